@@ -1,0 +1,198 @@
+/*
+ * augtree.h -- C interface of the prompt-sharing tree-attention library for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library computes, on one GPU, the attention part of the update-stage
+ * replay of a batch of prompt-response trees T = (P, {R_i}, i = 1..G)
+ * (Sec. 3.1 of the paper): one causal prefill of every shared prompt, the
+ * replay of every response branch against [shared prompt KV | own causal
+ * response KV] (Eq. 1), and the exact backward pass in which the prompt KV
+ * gradient is the sum over all branches (Eq. 2) and is then carried back
+ * through the prefill.
+ *
+ * Conventions that hold for every entry point
+ *  - Tensors are DEVICE pointers owned by the caller, bf16 unless stated,
+ *    laid out [tokens, heads, head_dim] with head_dim contiguous.  Prompt
+ *    tokens of all groups are packed back to back in group order; response
+ *    tokens are packed group-major, then branch order.  No padding, no
+ *    alignment requirement on the lengths; base pointers 16-byte aligned.
+ *  - LSE tensors are fp32 [H_q, tokens]: natural log of the sum of
+ *    exponentials of the scaled scores (m + ln l of the (m, l, O_acc) state of
+ *    Sec. 3.3).
+ *  - Query head h reads KV head h / (H_q / H_kv).
+ *  - Row a of a sequence sees keys b <= a (inclusive diagonal).
+ *  - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous; they
+ *    return after enqueueing.  Nothing is allocated or freed per call.
+ *  - Every function returns AUGTREE_OK (0) or a negative augtree_status code;
+ *    the library never aborts, traps or throws.  Errors detected on the
+ *    device (a bounded wait that ran out) are recorded in a status word that
+ *    augtree_last_device_status reads back.
+ *  - The descriptor arrays are HOST memory and are only read during
+ *    augtree_plan_create.
+ */
+#ifndef AUGTREE_H_
+#define AUGTREE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AUGTREE_VERSION 1u
+
+typedef enum {
+  AUGTREE_OK = 0,
+  AUGTREE_ERR_INVALID_ARG = -1, /* null pointer, non-positive length, bad struct size   */
+  AUGTREE_ERR_UNSUPPORTED = -2, /* head_dim not 64/128, h_q % h_kv != 0, sizes too big  */
+  AUGTREE_ERR_WORKSPACE = -3,   /* workspace pointer null or too small                  */
+  AUGTREE_ERR_CUDA = -4,        /* a CUDA runtime or driver call failed                 */
+  AUGTREE_ERR_TIMEOUT = -5,     /* a device-side wait gave up (status word)             */
+  AUGTREE_ERR_INTERNAL = -6
+} augtree_status;
+
+/* flags */
+#define AUGTREE_FLAG_ZERO_PROMPT_GRAD 1u /* replay_bwd clears dkp_acc/dvp_acc before accumulating */
+
+/*
+ * Packed group descriptor (host, plain data).  One entry per replay tree
+ * ("group"): its prompt length P_g >= 1, its branch count G_g >= 0 and, in
+ * branch_len, the G_g response lengths R_{g,i} >= 1 of every group one after
+ * another (Sec. 3.1: T = (P, {R_i})).  G_g = 0 describes a prompt with no
+ * responses; a batch of such groups is the flattened no-reuse baseline when
+ * each "prompt" is one linear sequence [P; R_i] (the ordinary causal pass of
+ * Sec. 3.4, b = 0).
+ */
+typedef struct {
+  uint32_t struct_size;       /* sizeof(augtree_desc_t)                                  */
+  uint32_t version;           /* AUGTREE_VERSION                                         */
+  int32_t n_groups;
+  const int32_t *prompt_len;  /* [n_groups]                                       (host) */
+  const int32_t *n_branches;  /* [n_groups]                                       (host) */
+  const int32_t *branch_len;  /* [sum n_branches], group-major                    (host) */
+  int32_t h_q, h_kv, head_dim;/* head_dim in {64, 128}                                   */
+  float softmax_scale;        /* 0 => 1/sqrt(head_dim)  (Sec. 2.2)                       */
+  uint32_t flags;
+  int32_t n_lanes;            /* replay lanes = persistent CTAs; 0 => SM count of device */
+  int32_t kv_splits;          /* prompt-KV shards per query tile in replay_fwd; 0/1 none */
+} augtree_desc_t;
+
+typedef struct augtree_plan augtree_plan_t;
+
+/* Tables returned by augtree_plan_metadata (all int32). */
+enum {
+  AUGTREE_TBL_CU_PROMPT = 0,      /* [n_groups+1] prefix sums of prompt_len                 */
+  AUGTREE_TBL_CU_BRANCH = 1,      /* [n_groups+1] prefix sums of n_branches                 */
+  AUGTREE_TBL_CU_RESPONSE = 2,    /* [n_branches+1] prefix sums of branch_len               */
+  AUGTREE_TBL_PREFILL_FWD_ITEMS = 3, AUGTREE_TBL_PREFILL_FWD_LANE_PTR = 4, AUGTREE_TBL_PREFILL_FWD_ORDER = 5,
+  AUGTREE_TBL_REPLAY_FWD_ITEMS = 6,  AUGTREE_TBL_REPLAY_FWD_LANE_PTR = 7,  AUGTREE_TBL_REPLAY_FWD_ORDER = 8,
+  AUGTREE_TBL_REPLAY_BWD_ITEMS = 9,  AUGTREE_TBL_REPLAY_BWD_LANE_PTR = 10, AUGTREE_TBL_REPLAY_BWD_ORDER = 11,
+  AUGTREE_TBL_PREFILL_BWD_ITEMS = 12, AUGTREE_TBL_PREFILL_BWD_LANE_PTR = 13, AUGTREE_TBL_PREFILL_BWD_ORDER = 14,
+  AUGTREE_TBL_REPLAY_SEGMENTS = 15,  /* [n_branches][2] {first response token, length}      */
+  AUGTREE_TBL_PREFILL_SEGMENTS = 16, /* [n_groups][2]   {first prompt token, length}        */
+  AUGTREE_TBL_GROUP_SPLITS = 17,     /* [n_groups] prompt-KV shards actually used           */
+  AUGTREE_TBL_COUNT = 18
+};
+#define AUGTREE_FWD_ITEM_INTS 12
+#define AUGTREE_BWD_ITEM_INTS 8
+
+/*
+ * Pack and schedule (host).  Validates the descriptor, builds the prefix sums
+ * and, for each of the four kernels, the list of work items and their
+ * assignment to `n_lanes` replay lanes: items weighted by their valid Q-KV
+ * tile count are placed largest first on the least loaded lane (the balanced
+ * makespan assignment of Sec. 3.4, Eq. 6, in its greedy form with one round).
+ * With device >= 0 the tables are also copied to that device and a status
+ * word is allocated there; with device < 0 the plan is host-only (metadata
+ * queries work, launches return AUGTREE_ERR_INVALID_ARG) and n_lanes must be
+ * given.  This is the only entry point, with augtree_plan_destroy, that
+ * allocates or frees device memory.
+ */
+int augtree_plan_create(const augtree_desc_t *desc, int device, augtree_plan_t **out);
+int augtree_plan_destroy(augtree_plan_t *plan);
+
+/* Bytes of caller-provided scratch the forward and backward calls need. */
+int augtree_plan_workspace_bytes(const augtree_plan_t *plan, size_t *fwd_bytes, size_t *bwd_bytes);
+
+/*
+ * Copy one metadata table to host memory.  With host_dst == NULL only *bytes
+ * is set.  Otherwise *bytes is the capacity on entry and the size on return.
+ * Item layouts (int32 each):
+ *   forward item  [12]: q_tok0, q_pos0, q_rows, q_head, a_tok0, a_len, b_tok0,
+ *                       b_len, split, n_splits, weight, kv_head
+ *     a_* : unmasked key range (shared prompt KV, Eq. 1's KV_P), b_* : causal
+ *     key range of the query's own sequence, length already clipped to what
+ *     the tile's last row sees.
+ *   backward item [8] : kv_tok0, kv_pos0, kv_rows, kv_head, mode, seg0, nseg,
+ *                       weight;  mode 0 = causal inside one sequence, mode 1 =
+ *     shared prompt keys against every response query of the group (Eq. 2).
+ *   *_LANE_PTR [n_lanes+1], *_ORDER [n_items]: lane l runs the items
+ *     ORDER[LANE_PTR[l] .. LANE_PTR[l+1]) in that order.
+ */
+int augtree_plan_metadata(const augtree_plan_t *plan, int table_id, void *host_dst, size_t *bytes);
+
+/*
+ * Prompt prefill, forward (Sec. 3.2, "Shared prompt prefill pass"): causal
+ * attention of every prompt on itself.  k_p/v_p are only read and stay where
+ * they are for the replay calls.
+ *   q_p [sumP,H_q,d]  k_p,v_p [sumP,H_kv,d]  ->  o_p [sumP,H_q,d] bf16, lse_p [H_q,sumP] fp32
+ */
+int augtree_prefill_fwd(const augtree_plan_t *plan, const void *q_p, const void *k_p, const void *v_p,
+                        void *o_p, float *lse_p, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Response replay, forward (Sec. 3.2 "Response replay", Sec. 3.3): every
+ * response query attends to the shared prompt KV (unmasked) and to its own
+ * branch (causal); the partial softmax states of the parts are merged
+ * (the (+) of Sec. 3.3).  With kv_splits > 1 the prompt KV of a query tile is
+ * processed as independent shards whose states are merged by a second kernel.
+ *   q_r [sumR,H_q,d] k_r,v_r [sumR,H_kv,d] k_p,v_p -> o_r [sumR,H_q,d] bf16, lse_r [H_q,sumR] fp32
+ */
+int augtree_replay_fwd(const augtree_plan_t *plan, const void *q_r, const void *k_r, const void *v_r,
+                       const void *k_p, const void *v_p, void *o_r, float *lse_r,
+                       void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Response replay, backward (Sec. 3.2, "Exact many-to-one backward", Eq. 2).
+ * Inputs as the forward plus its outputs o_r, lse_r and the seed do_r.
+ * Outputs dq_r [sumR,H_q,d], dk_r, dv_r [sumR,H_kv,d] bf16.  The prompt-KV
+ * gradients of all branches and query heads are ADDED into the fp32
+ * accumulators dkp_acc, dvp_acc [sumP,H_kv,d], which the caller zeroes first
+ * (or sets AUGTREE_FLAG_ZERO_PROMPT_GRAD in the descriptor).  Each prompt-KV
+ * tile is owned by one lane, so this sum has a fixed order; dq_r is summed
+ * with fp32 atomics in scratch and rounded once.
+ */
+int augtree_replay_bwd(const augtree_plan_t *plan, const void *q_r, const void *k_r, const void *v_r,
+                       const void *k_p, const void *v_p, const void *o_r, const float *lse_r,
+                       const void *do_r, void *dq_r, void *dk_r, void *dv_r,
+                       float *dkp_acc, float *dvp_acc, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Prompt prefill, backward: the causal backward of augtree_prefill_fwd under
+ * the seed do_p.  Its dK/dV are ADDED to dkp_acc/dvp_acc, which after this
+ * call hold the final prompt-KV gradients (replay seeds + prefill graph,
+ * Sec. 3.2); call it after augtree_replay_bwd on the same stream.  dq_p is
+ * written; dk_p/dv_p (bf16 copies of the final accumulators) may be NULL.
+ */
+int augtree_prefill_bwd(const augtree_plan_t *plan, const void *q_p, const void *k_p, const void *v_p,
+                        const void *o_p, const float *lse_p, const void *do_p,
+                        float *dkp_acc, float *dvp_acc, void *dq_p, void *dk_p, void *dv_p,
+                        void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Synchronises the plan's device and reads the device status word: *status is
+ * AUGTREE_OK or AUGTREE_ERR_TIMEOUT; *detail (may be NULL) gets a code that
+ * names the wait that gave up.  The word is cleared by the read.
+ */
+int augtree_last_device_status(const augtree_plan_t *plan, int *status, int *detail);
+
+/* Number of kernel launches the library has enqueued since it was loaded. */
+long long augtree_launch_count(void);
+
+const char *augtree_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AUGTREE_H_ */

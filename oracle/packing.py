@@ -1,0 +1,129 @@
+"""Independent restatement of the pack-and-schedule metadata (test infrastructure only).
+
+Written from the rules, not from the library's source: the tests demand that
+the library's tables equal these bit for bit.
+
+Rules.  Tiles are 128 query rows by 128 keys.  A forward item is one (query
+tile, query head[, prompt-KV shard]); its weight is the number of KV tiles it
+visits.  A backward item is one (KV tile, KV head); its weight is the number of
+(query tile, query head) visits.  Items are listed in a canonical order, then
+assigned to lanes largest weight first (ties: lower id first), each to the lane
+with the least load so far (ties: lowest lane), following the balanced
+makespan assignment of Sec. 3.4 / Eq. 6 in its greedy form; a lane runs its
+items in ascending id.
+"""
+from __future__ import annotations
+
+import heapq
+
+import numpy as np
+
+TQ = TK = 128
+
+
+def _cdiv(a, b):
+    return -(-a // b)
+
+
+def prefix(xs):
+    out = [0]
+    for x in xs:
+        out.append(out[-1] + x)
+    return out
+
+
+def build_tables(prompt_len, branch_len, h_q, h_kv, kv_splits=1):
+    rep = h_q // h_kv
+    cu_p = prefix(prompt_len)
+    cu_b = prefix([len(b) for b in branch_len])
+    flat = [r for b in branch_len for r in b]
+    cu_r = prefix(flat)
+    kv_splits = max(1, kv_splits)
+    pf, rf, rb, pb, gsplits = [], [], [], [], []
+    for g, P in enumerate(prompt_len):
+        p0 = cu_p[g]
+        na = _cdiv(P, TK)
+        shard_tiles = _cdiv(na, min(kv_splits, na))
+        ns = _cdiv(na, shard_tiles)
+        gsplits.append(ns)
+        for c in range(h_kv):
+            for t in range(_cdiv(P, TQ)):
+                rows = min(TQ, P - t * TQ)
+                vis = t * TQ + rows
+                for j in range(rep):
+                    pf.append([p0 + t * TQ, t * TQ, rows, c * rep + j, 0, 0, p0, vis, 0, 1, _cdiv(vis, TK), c])
+            for bi in range(cu_b[g], cu_b[g + 1]):
+                R, r0 = flat[bi], cu_r[bi]
+                for t in range(_cdiv(R, TQ)):
+                    rows = min(TQ, R - t * TQ)
+                    vis = t * TQ + rows
+                    for j in range(rep):
+                        for s in range(ns):
+                            a0 = s * shard_tiles * TK
+                            alen = min(P - a0, shard_tiles * TK)
+                            bl = vis if s == ns - 1 else 0
+                            rf.append([r0 + t * TQ, t * TQ, rows, c * rep + j, p0 + a0, alen, r0, bl, s, ns,
+                                       _cdiv(alen, TK) + _cdiv(bl, TK), c])
+            b0, b1 = cu_b[g], cu_b[g + 1]
+            if b1 > b0:
+                visits = sum(_cdiv(flat[bi], TQ) * rep for bi in range(b0, b1))
+                for t in range(_cdiv(P, TK)):
+                    rb.append([p0 + t * TK, t * TK, min(TK, P - t * TK), c, 1, b0, b1 - b0, visits])
+            for bi in range(b0, b1):
+                R, r0 = flat[bi], cu_r[bi]
+                for t in range(_cdiv(R, TK)):
+                    rb.append([r0 + t * TK, t * TK, min(TK, R - t * TK), c, 0, bi, 1, (_cdiv(R, TQ) - t) * rep])
+            for t in range(_cdiv(P, TK)):
+                pb.append([p0 + t * TK, t * TK, min(TK, P - t * TK), c, 0, g, 1, (_cdiv(P, TQ) - t) * rep])
+    arr = lambda x, w: np.asarray(x, dtype=np.int32).reshape(-1, w)
+    return {
+        "cu_p": np.asarray(cu_p, np.int32), "cu_b": np.asarray(cu_b, np.int32), "cu_r": np.asarray(cu_r, np.int32),
+        "prefill_fwd": arr(pf, 12), "replay_fwd": arr(rf, 12), "replay_bwd": arr(rb, 8), "prefill_bwd": arr(pb, 8),
+        "group_splits": np.asarray(gsplits, np.int32),
+        "seg_replay": np.asarray([[cu_r[i], flat[i]] for i in range(len(flat))], np.int32).reshape(-1, 2),
+        "seg_prefill": np.asarray([[cu_p[g], prompt_len[g]] for g in range(len(prompt_len))], np.int32).reshape(-1, 2),
+    }
+
+
+def assign_lanes(weights, n_lanes):
+    """Largest-first greedy assignment.  Returns (lane_ptr [n_lanes+1], order [n])."""
+    ids = sorted(range(len(weights)), key=lambda i: (-int(weights[i]), i))
+    heap = [(0, l) for l in range(n_lanes)]
+    heapq.heapify(heap)
+    lanes = [[] for _ in range(n_lanes)]
+    for i in ids:
+        load, l = heapq.heappop(heap)
+        lanes[l].append(i)
+        heapq.heappush(heap, (load + int(weights[i]), l))
+    order, ptr = [], [0]
+    for l in range(n_lanes):
+        order += sorted(lanes[l])
+        ptr.append(len(order))
+    return np.asarray(ptr, np.int32), np.asarray(order, np.int32)
+
+
+def makespan(weights, lane_ptr, order):
+    w = np.asarray(weights)
+    return max(int(w[order[lane_ptr[l]:lane_ptr[l + 1]]].sum()) for l in range(len(lane_ptr) - 1))
+
+
+def brute_force_makespan(weights, n_lanes):
+    """Optimal makespan by exhaustive assignment (tiny inputs only)."""
+    best = [sum(weights)]
+    loads = [0] * n_lanes
+
+    def rec(i):
+        if i == len(weights):
+            best[0] = min(best[0], max(loads))
+            return
+        seen = set()
+        for l in range(n_lanes):
+            if loads[l] in seen:
+                continue
+            seen.add(loads[l])
+            loads[l] += weights[i]
+            if max(loads) < best[0]:
+                rec(i + 1)
+            loads[l] -= weights[i]
+    rec(0)
+    return best[0]

@@ -1,0 +1,163 @@
+"""ctypes binding of libaugtree.so: argument marshalling only.
+
+Every step of the path runs inside the library's kernels.  PyTorch appears only
+as the owner of device memory and of the current stream.  Importing this module
+raises if the library has not been built (there is no CPU fallback):
+run `python -m paper_2609_33133_b200.build`.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libaugtree.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_33133_b200.build`")
+lib = C.CDLL(LIB_PATH)
+
+FLAG_ZERO_PROMPT_GRAD = 1
+FWD_ITEM_INTS, BWD_ITEM_INTS = 12, 8
+(TBL_CU_PROMPT, TBL_CU_BRANCH, TBL_CU_RESPONSE, TBL_PREFILL_FWD_ITEMS, TBL_PREFILL_FWD_LANE_PTR, TBL_PREFILL_FWD_ORDER,
+ TBL_REPLAY_FWD_ITEMS, TBL_REPLAY_FWD_LANE_PTR, TBL_REPLAY_FWD_ORDER, TBL_REPLAY_BWD_ITEMS, TBL_REPLAY_BWD_LANE_PTR,
+ TBL_REPLAY_BWD_ORDER, TBL_PREFILL_BWD_ITEMS, TBL_PREFILL_BWD_LANE_PTR, TBL_PREFILL_BWD_ORDER, TBL_REPLAY_SEGMENTS,
+ TBL_PREFILL_SEGMENTS, TBL_GROUP_SPLITS) = range(18)
+
+EXPORTS = ["augtree_plan_create", "augtree_plan_destroy", "augtree_plan_workspace_bytes", "augtree_plan_metadata",
+           "augtree_prefill_fwd", "augtree_replay_fwd", "augtree_replay_bwd", "augtree_prefill_bwd",
+           "augtree_last_device_status", "augtree_launch_count", "augtree_status_string"]
+
+
+class Desc(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("version", C.c_uint32), ("n_groups", C.c_int32),
+                ("prompt_len", C.POINTER(C.c_int32)), ("n_branches", C.POINTER(C.c_int32)),
+                ("branch_len", C.POINTER(C.c_int32)), ("h_q", C.c_int32), ("h_kv", C.c_int32),
+                ("head_dim", C.c_int32), ("softmax_scale", C.c_float), ("flags", C.c_uint32),
+                ("n_lanes", C.c_int32), ("kv_splits", C.c_int32)]
+
+
+_vp, _sz = C.c_void_p, C.c_size_t
+lib.augtree_plan_create.argtypes = [C.POINTER(Desc), C.c_int, C.POINTER(_vp)]
+lib.augtree_plan_destroy.argtypes = [_vp]
+lib.augtree_plan_workspace_bytes.argtypes = [_vp, C.POINTER(_sz), C.POINTER(_sz)]
+lib.augtree_plan_metadata.argtypes = [_vp, C.c_int, _vp, C.POINTER(_sz)]
+lib.augtree_prefill_fwd.argtypes = [_vp] + [_vp] * 5 + [_vp, _sz, _vp]
+lib.augtree_replay_fwd.argtypes = [_vp] + [_vp] * 7 + [_vp, _sz, _vp]
+lib.augtree_replay_bwd.argtypes = [_vp] + [_vp] * 13 + [_vp, _sz, _vp]
+lib.augtree_prefill_bwd.argtypes = [_vp] + [_vp] * 11 + [_vp, _sz, _vp]
+lib.augtree_last_device_status.argtypes = [_vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+lib.augtree_launch_count.restype = C.c_longlong
+lib.augtree_status_string.restype = C.c_char_p
+lib.augtree_status_string.argtypes = [C.c_int]
+
+
+class AugtreeError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {lib.augtree_status_string(code).decode()} ({code})")
+
+
+def _check(code, where):
+    if code != 0:
+        raise AugtreeError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def launch_count() -> int:
+    return int(lib.augtree_launch_count())
+
+
+class Plan:
+    """Owns an augtree_plan_t.  device=None builds a host-only plan (metadata queries only)."""
+
+    def __init__(self, prompt_len, branch_len, h_q, h_kv, head_dim, *, device=0, softmax_scale=0.0, flags=0,
+                 n_lanes=0, kv_splits=0):
+        self.prompt_len = [int(x) for x in prompt_len]
+        self.branch_len = [[int(x) for x in b] for b in branch_len]
+        self.h_q, self.h_kv, self.head_dim = h_q, h_kv, head_dim
+        self.total_p = sum(self.prompt_len)
+        self.total_r = sum(sum(b) for b in self.branch_len)
+        n = len(self.prompt_len)
+        flat = [r for b in self.branch_len for r in b]
+        self._pl = (C.c_int32 * n)(*self.prompt_len)
+        self._nb = (C.c_int32 * n)(*[len(b) for b in self.branch_len])
+        self._bl = (C.c_int32 * max(len(flat), 1))(*flat)
+        d = Desc(C.sizeof(Desc), 1, n, self._pl, self._nb, self._bl, h_q, h_kv, head_dim, softmax_scale, flags,
+                 n_lanes, kv_splits)
+        self._h = C.c_void_p()
+        self.device = device
+        _check(lib.augtree_plan_create(C.byref(d), -1 if device is None else int(device), C.byref(self._h)), "plan_create")
+        f, b = _sz(), _sz()
+        _check(lib.augtree_plan_workspace_bytes(self._h, C.byref(f), C.byref(b)), "workspace_bytes")
+        self.ws_fwd_bytes, self.ws_bwd_bytes = f.value, b.value
+
+    def __del__(self):
+        h = getattr(self, "_h", None)
+        if h is not None and h.value:
+            lib.augtree_plan_destroy(h)
+            self._h = None
+
+    def metadata(self, table_id) -> np.ndarray:
+        n = _sz()
+        _check(lib.augtree_plan_metadata(self._h, table_id, None, C.byref(n)), "plan_metadata")
+        out = np.zeros(n.value // 4, dtype=np.int32)
+        _check(lib.augtree_plan_metadata(self._h, table_id, out.ctypes.data_as(C.c_void_p), C.byref(n)), "plan_metadata")
+        return out
+
+    @staticmethod
+    def _stream():
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+    def prefill_fwd(self, q_p, k_p, v_p, o_p, lse_p, ws=None):
+        _check(lib.augtree_prefill_fwd(self._h, _ptr(q_p), _ptr(k_p), _ptr(v_p), _ptr(o_p), _ptr(lse_p), _ptr(ws),
+                                       0 if ws is None else ws.numel() * ws.element_size(), self._stream()), "prefill_fwd")
+
+    def replay_fwd(self, q_r, k_r, v_r, k_p, v_p, o_r, lse_r, ws=None):
+        _check(lib.augtree_replay_fwd(self._h, _ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(k_p), _ptr(v_p), _ptr(o_r),
+                                      _ptr(lse_r), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                      self._stream()), "replay_fwd")
+
+    def replay_bwd(self, q_r, k_r, v_r, k_p, v_p, o_r, lse_r, do_r, dq_r, dk_r, dv_r, dkp_acc, dvp_acc, ws):
+        _check(lib.augtree_replay_bwd(self._h, _ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(k_p), _ptr(v_p), _ptr(o_r),
+                                      _ptr(lse_r), _ptr(do_r), _ptr(dq_r), _ptr(dk_r), _ptr(dv_r), _ptr(dkp_acc),
+                                      _ptr(dvp_acc), _ptr(ws), ws.numel() * ws.element_size(), self._stream()), "replay_bwd")
+
+    def prefill_bwd(self, q_p, k_p, v_p, o_p, lse_p, do_p, dkp_acc, dvp_acc, dq_p, dk_p=None, dv_p=None, ws=None):
+        _check(lib.augtree_prefill_bwd(self._h, _ptr(q_p), _ptr(k_p), _ptr(v_p), _ptr(o_p), _ptr(lse_p), _ptr(do_p),
+                                       _ptr(dkp_acc), _ptr(dvp_acc), _ptr(dq_p), _ptr(dk_p), _ptr(dv_p), _ptr(ws),
+                                       0 if ws is None else ws.numel() * ws.element_size(), self._stream()), "prefill_bwd")
+
+    def device_status(self):
+        s, d = C.c_int(), C.c_int()
+        _check(lib.augtree_last_device_status(self._h, C.byref(s), C.byref(d)), "last_device_status")
+        return s.value, d.value
+
+
+def alloc_outputs(plan: Plan, device="cuda"):
+    """Device buffers for one forward + backward pass (allocation only)."""
+    hq, hkv, d = plan.h_q, plan.h_kv, plan.head_dim
+    bf, f32 = torch.bfloat16, torch.float32
+    e = lambda *s, dt=bf: torch.empty(s, device=device, dtype=dt)
+    tp, tr = plan.total_p, plan.total_r
+    return {
+        "o_p": e(tp, hq, d), "lse_p": e(hq, tp, dt=f32), "o_r": e(tr, hq, d), "lse_r": e(hq, tr, dt=f32),
+        "dq_p": e(tp, hq, d), "dq_r": e(tr, hq, d), "dk_r": e(tr, hkv, d), "dv_r": e(tr, hkv, d),
+        "dk_p": torch.zeros((tp, hkv, d), device=device, dtype=f32), "dv_p": torch.zeros((tp, hkv, d), device=device, dtype=f32),
+        "ws": torch.empty(max(plan.ws_fwd_bytes, plan.ws_bwd_bytes, 256), device=device, dtype=torch.uint8),
+    }
+
+
+def run_forward_backward(plan: Plan, t, out):
+    """The whole hot path, in call order, on the current stream: 4 entry points."""
+    plan.prefill_fwd(t["q_p"], t["k_p"], t["v_p"], out["o_p"], out["lse_p"], out["ws"])
+    plan.replay_fwd(t["q_r"], t["k_r"], t["v_r"], t["k_p"], t["v_p"], out["o_r"], out["lse_r"], out["ws"])
+    plan.replay_bwd(t["q_r"], t["k_r"], t["v_r"], t["k_p"], t["v_p"], out["o_r"], out["lse_r"], t["do_r"],
+                    out["dq_r"], out["dk_r"], out["dv_r"], out["dk_p"], out["dv_p"], out["ws"])
+    plan.prefill_bwd(t["q_p"], t["k_p"], t["v_p"], out["o_p"], out["lse_p"], t["do_p"], out["dk_p"], out["dv_p"],
+                     out["dq_p"], None, None, out["ws"])

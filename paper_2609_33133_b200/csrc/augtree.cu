@@ -1,0 +1,405 @@
+// C-ABI entry points: plan lifetime, tensor-map encoding and kernel launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstring>
+#include <mutex>
+#include <new>
+
+#include "bwd_kernel.cuh"
+#include "fwd_kernel.cuh"
+#include "plan.h"
+
+using namespace augtree;
+
+namespace {
+
+std::atomic<long long> g_launches{0};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  });
+  return fn;
+}
+
+// Tensor map over a packed [tokens, heads, d] bf16 tensor; one box = 128 tokens
+// of one head, 64 elements (128 bytes) wide, written to shared memory with the
+// 128-byte swizzle.  Rows past the end of the tensor read as zero.
+int make_map(CUtensorMap *m, const void *ptr, long long tokens, int heads, int d) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return AUGTREE_ERR_CUDA;
+  if (tokens < 1) tokens = 1;
+  const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)heads, (cuuint64_t)tokens};
+  const cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)heads * d * 2};
+  const cuuint32_t box[3] = {64, 1, 128};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+size_t al256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+int upload(const std::vector<int32_t> &h, int32_t **d) {
+  *d = nullptr;
+  const size_t bytes = (h.size() ? h.size() : 1) * sizeof(int32_t);
+  if (cudaMalloc(d, bytes) != cudaSuccess) return AUGTREE_ERR_CUDA;
+  if (!h.empty() && cudaMemcpy(*d, h.data(), h.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
+    return AUGTREE_ERR_CUDA;
+  return AUGTREE_OK;
+}
+
+int upload_sched(Sched &s, int n_lanes) {
+  std::vector<int32_t> sorted(s.items.size());
+  for (size_t i = 0; i < s.order.size(); ++i)
+    std::memcpy(&sorted[i * s.item_ints], &s.items[(size_t)s.order[i] * s.item_ints], s.item_ints * sizeof(int32_t));
+  int r = upload(sorted, &s.d_items);
+  if (r) return r;
+  (void)n_lanes;
+  return upload(s.lane_ptr, &s.d_lane_ptr);
+}
+
+template <int D>
+int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long q_tok, const void *ka, const void *va,
+               long long a_tok, const void *kb, const void *vb, long long b_tok, void *o, float *lse, float *part_o,
+               float *part_lse, cudaStream_t st) {
+  if (s.n_items() == 0) return AUGTREE_OK;
+  CUtensorMap mq, mka, mva, mkb, mvb;
+  int r;
+  if ((r = make_map(&mq, q, q_tok, pl->h_q, D))) return r;
+  if ((r = make_map(&mka, ka, a_tok, pl->h_kv, D))) return r;
+  if ((r = make_map(&mva, va, a_tok, pl->h_kv, D))) return r;
+  if ((r = make_map(&mkb, kb, b_tok, pl->h_kv, D))) return r;
+  if ((r = make_map(&mvb, vb, b_tok, pl->h_kv, D))) return r;
+  FwdParams p;
+  p.items = s.d_items; p.lane_ptr = s.d_lane_ptr;
+  p.o = static_cast<__nv_bfloat16 *>(o); p.lse = lse; p.part_o = part_o; p.part_lse = part_lse;
+  p.n_tok = q_tok; p.h_q = pl->h_q; p.scale_log2 = pl->scale * 1.4426950408889634f; p.status = pl->d_status;
+  static bool attr_set[2] = {false, false};
+  if (!attr_set[D / 128]) {
+    if (cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kBytes) != cudaSuccess)
+      return AUGTREE_ERR_CUDA;
+    attr_set[D / 128] = true;
+  }
+  fwd_kernel<D><<<pl->n_lanes, kFwdThreads, FwdSmem<D>::kBytes, st>>>(mq, mka, mva, mkb, mvb, p);
+  ++g_launches;
+  return cudaGetLastError() == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+}
+
+struct BwdArgs {
+  const void *q, *d_o, *o;
+  const float *lse;
+  long long q_tok;
+  const void *k0, *v0; long long kv0_tok;  // mode-0 K/V tensor (the queries' own sequence)
+  const void *k1, *v1; long long kv1_tok;  // mode-1 K/V tensor (shared prompt)
+  void *dq; void *dk_out, *dv_out;
+  float *dk_acc, *dv_acc;
+  int causal_fp32;
+  const int32_t *d_segs;
+};
+
+template <int D>
+int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *ws, cudaStream_t st) {
+  const size_t hq = pl->h_q;
+  const size_t n_el = (size_t)a.q_tok * hq * D;
+  if (n_el == 0) return AUGTREE_OK;
+  uint8_t *w = static_cast<uint8_t *>(ws);
+  float *dq_acc = reinterpret_cast<float *>(w);
+  // region sizes must match build_plan_host: sized for max(total_p, total_r)
+  const size_t tmax = (size_t)(pl->total_p > pl->total_r ? pl->total_p : pl->total_r);
+  float *delta = reinterpret_cast<float *>(w + al256(tmax * hq * D * 4));
+  float *lse2 = reinterpret_cast<float *>(w + al256(tmax * hq * D * 4) + al256(tmax * hq * 4));
+  if (cudaMemsetAsync(dq_acc, 0, n_el * 4, st) != cudaSuccess) return AUGTREE_ERR_CUDA;
+  {
+    const long long warps = a.q_tok * (long long)hq;
+    const int threads = 256;
+    const long long blocks = (warps * 32 + threads - 1) / threads;
+    bwd_preprocess_kernel<D><<<(unsigned)blocks, threads, 0, st>>>(
+        static_cast<const __nv_bfloat16 *>(a.o), static_cast<const __nv_bfloat16 *>(a.d_o), a.lse, delta, lse2, a.q_tok,
+        pl->h_q);
+    ++g_launches;
+  }
+  if (s.n_items() > 0) {
+    CUtensorMap mq, mdo, mk0, mv0, mk1, mv1;
+    int r;
+    if ((r = make_map(&mq, a.q, a.q_tok, pl->h_q, D))) return r;
+    if ((r = make_map(&mdo, a.d_o, a.q_tok, pl->h_q, D))) return r;
+    if ((r = make_map(&mk0, a.k0, a.kv0_tok, pl->h_kv, D))) return r;
+    if ((r = make_map(&mv0, a.v0, a.kv0_tok, pl->h_kv, D))) return r;
+    if ((r = make_map(&mk1, a.k1, a.kv1_tok, pl->h_kv, D))) return r;
+    if ((r = make_map(&mv1, a.v1, a.kv1_tok, pl->h_kv, D))) return r;
+    BwdParams p;
+    p.items = s.d_items; p.lane_ptr = s.d_lane_ptr; p.segs = a.d_segs; p.lse2 = lse2; p.delta = delta; p.dq_acc = dq_acc;
+    p.dk_out = static_cast<__nv_bfloat16 *>(a.dk_out); p.dv_out = static_cast<__nv_bfloat16 *>(a.dv_out);
+    p.dk_acc = a.dk_acc; p.dv_acc = a.dv_acc; p.n_tok = a.q_tok; p.h_q = pl->h_q; p.h_kv = pl->h_kv;
+    p.causal_fp32 = a.causal_fp32; p.scale = pl->scale; p.scale_log2 = pl->scale * 1.4426950408889634f;
+    p.status = pl->d_status;
+    static bool attr_set[2] = {false, false};
+    if (!attr_set[D / 128]) {
+      if (cudaFuncSetAttribute(bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kBytes) != cudaSuccess)
+        return AUGTREE_ERR_CUDA;
+      attr_set[D / 128] = true;
+    }
+    bwd_kernel<D><<<pl->n_lanes, kBwdThreads, BwdSmem<D>::kBytes, st>>>(mq, mdo, mk0, mv0, mk1, mv1, p);
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) return AUGTREE_ERR_CUDA;
+  }
+  {
+    const long long n4 = (long long)(n_el / 4);
+    cast_bf16_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(dq_acc, static_cast<__nv_bfloat16 *>(a.dq), n4);
+    ++g_launches;
+  }
+  return cudaGetLastError() == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+}
+
+int check_plan(const augtree_plan *pl) {
+  if (!pl || pl->device < 0 || pl->n_lanes < 1) return AUGTREE_ERR_INVALID_ARG;
+  return AUGTREE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int augtree_plan_create(const augtree_desc_t *desc, int device, augtree_plan_t **out) {
+  if (!out) return AUGTREE_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!desc) return AUGTREE_ERR_INVALID_ARG;
+  augtree_plan *pl = new (std::nothrow) augtree_plan();
+  if (!pl) return AUGTREE_ERR_INTERNAL;
+  augtree_desc_t d = *desc;
+  if (device >= 0 && d.struct_size == sizeof(augtree_desc_t) && d.n_lanes == 0) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1) {
+      delete pl;
+      return AUGTREE_ERR_CUDA;
+    }
+    d.n_lanes = sms;
+  }
+  if (device < 0 && d.struct_size == sizeof(augtree_desc_t) && d.n_lanes < 1) { delete pl; return AUGTREE_ERR_INVALID_ARG; }
+  int r = AUGTREE_ERR_INTERNAL;
+  try {
+    r = build_plan_host(&d, pl);
+  } catch (...) {
+    r = AUGTREE_ERR_INTERNAL;
+  }
+  if (r) { delete pl; return r; }
+  pl->device = device;
+  if (device >= 0) {
+    int prev = 0;
+    cudaGetDevice(&prev);
+    r = cudaSetDevice(device) == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+    for (int k = 0; k < SCHED_COUNT && !r; ++k) r = upload_sched(pl->sched[k], pl->n_lanes);
+    if (!r) r = upload(pl->seg_replay, &pl->d_seg_replay);
+    if (!r) r = upload(pl->seg_prefill, &pl->d_seg_prefill);
+    if (!r) r = upload(pl->branch_group, &pl->d_branch_group);
+    if (!r) r = upload(pl->group_splits, &pl->d_group_splits);
+    if (!r) r = upload(pl->cu_r, &pl->d_cu_r);
+    if (!r) {
+      if (cudaMalloc(&pl->d_status, 2 * sizeof(int)) != cudaSuccess || cudaMemset(pl->d_status, 0, 2 * sizeof(int)) != cudaSuccess)
+        r = AUGTREE_ERR_CUDA;
+    }
+    cudaSetDevice(prev);
+    if (r) { augtree_plan_destroy(pl); return r; }
+  }
+  *out = pl;
+  return AUGTREE_OK;
+}
+
+int augtree_plan_destroy(augtree_plan_t *pl) {
+  if (!pl) return AUGTREE_ERR_INVALID_ARG;
+  if (pl->device >= 0) {
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(pl->device);
+    for (int k = 0; k < SCHED_COUNT; ++k) { cudaFree(pl->sched[k].d_items); cudaFree(pl->sched[k].d_lane_ptr); }
+    cudaFree(pl->d_seg_replay); cudaFree(pl->d_seg_prefill); cudaFree(pl->d_branch_group); cudaFree(pl->d_group_splits);
+    cudaFree(pl->d_cu_r); cudaFree(pl->d_status);
+    cudaSetDevice(prev);
+  }
+  delete pl;
+  return AUGTREE_OK;
+}
+
+int augtree_plan_workspace_bytes(const augtree_plan_t *pl, size_t *fwd, size_t *bwd) {
+  if (!pl) return AUGTREE_ERR_INVALID_ARG;
+  if (fwd) *fwd = pl->ws_fwd;
+  if (bwd) *bwd = pl->ws_bwd;
+  return AUGTREE_OK;
+}
+
+int augtree_plan_metadata(const augtree_plan_t *pl, int table_id, void *host_dst, size_t *bytes) {
+  if (!pl || !bytes) return AUGTREE_ERR_INVALID_ARG;
+  const std::vector<int32_t> *v = nullptr;
+  switch (table_id) {
+    case AUGTREE_TBL_CU_PROMPT: v = &pl->cu_p; break;
+    case AUGTREE_TBL_CU_BRANCH: v = &pl->cu_b; break;
+    case AUGTREE_TBL_CU_RESPONSE: v = &pl->cu_r; break;
+    case AUGTREE_TBL_REPLAY_SEGMENTS: v = &pl->seg_replay; break;
+    case AUGTREE_TBL_PREFILL_SEGMENTS: v = &pl->seg_prefill; break;
+    case AUGTREE_TBL_GROUP_SPLITS: v = &pl->group_splits; break;
+    default:
+      if (table_id >= AUGTREE_TBL_PREFILL_FWD_ITEMS && table_id <= AUGTREE_TBL_PREFILL_BWD_ORDER) {
+        const Sched &s = pl->sched[(table_id - 3) / 3];
+        const int which = (table_id - 3) % 3;
+        v = which == 0 ? &s.items : which == 1 ? &s.lane_ptr : &s.order;
+      }
+  }
+  if (!v) return AUGTREE_ERR_INVALID_ARG;
+  const size_t need = v->size() * sizeof(int32_t);
+  if (!host_dst) { *bytes = need; return AUGTREE_OK; }
+  if (*bytes < need) { *bytes = need; return AUGTREE_ERR_INVALID_ARG; }
+  if (need) std::memcpy(host_dst, v->data(), need);
+  *bytes = need;
+  return AUGTREE_OK;
+}
+
+int augtree_prefill_fwd(const augtree_plan_t *pl, const void *q_p, const void *k_p, const void *v_p, void *o_p,
+                        float *lse_p, void *ws, size_t ws_bytes, void *stream) {
+  (void)ws; (void)ws_bytes;
+  int r = check_plan(pl);
+  if (r) return r;
+  if (!q_p || !k_p || !v_p || !o_p || !lse_p) return AUGTREE_ERR_INVALID_ARG;
+  if (!aligned16(q_p) || !aligned16(k_p) || !aligned16(v_p) || !aligned16(o_p)) return AUGTREE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Sched &s = pl->sched[SCHED_PREFILL_FWD];
+  if (pl->head_dim == 128)
+    return launch_fwd<128>(pl, s, q_p, pl->total_p, k_p, v_p, pl->total_p, k_p, v_p, pl->total_p, o_p, lse_p, nullptr, nullptr, st);
+  return launch_fwd<64>(pl, s, q_p, pl->total_p, k_p, v_p, pl->total_p, k_p, v_p, pl->total_p, o_p, lse_p, nullptr, nullptr, st);
+}
+
+int augtree_replay_fwd(const augtree_plan_t *pl, const void *q_r, const void *k_r, const void *v_r, const void *k_p,
+                       const void *v_p, void *o_r, float *lse_r, void *ws, size_t ws_bytes, void *stream) {
+  int r = check_plan(pl);
+  if (r) return r;
+  if (pl->total_r == 0) return AUGTREE_OK;
+  if (!q_r || !k_r || !v_r || !k_p || !v_p || !o_r || !lse_r) return AUGTREE_ERR_INVALID_ARG;
+  if (!aligned16(q_r) || !aligned16(k_r) || !aligned16(v_r) || !aligned16(k_p) || !aligned16(v_p) || !aligned16(o_r))
+    return AUGTREE_ERR_INVALID_ARG;
+  float *part_o = nullptr, *part_lse = nullptr;
+  if (pl->max_splits > 1) {
+    if (!ws || ws_bytes < pl->ws_fwd || !aligned16(ws)) return AUGTREE_ERR_WORKSPACE;
+    part_o = static_cast<float *>(ws);
+    part_lse = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) +
+                                         al256((size_t)pl->max_splits * (size_t)pl->total_r * pl->h_q * pl->head_dim * 4));
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Sched &s = pl->sched[SCHED_REPLAY_FWD];
+  if (pl->head_dim == 128)
+    r = launch_fwd<128>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, o_r, lse_r, part_o, part_lse, st);
+  else
+    r = launch_fwd<64>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, o_r, lse_r, part_o, part_lse, st);
+  if (r || pl->max_splits == 1) return r;
+  // groups that ended up with one shard wrote their final output directly; the
+  // merge kernel only touches tokens whose group has more than one shard
+  const long long warps = pl->total_r * (long long)pl->h_q;
+  const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
+  if (pl->head_dim == 128)
+    combine_kernel<128><<<blocks, 256, 0, st>>>(part_o, part_lse, pl->d_cu_r, pl->d_branch_group, pl->d_group_splits,
+                                                pl->n_branches, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q);
+  else
+    combine_kernel<64><<<blocks, 256, 0, st>>>(part_o, part_lse, pl->d_cu_r, pl->d_branch_group, pl->d_group_splits,
+                                               pl->n_branches, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q);
+  ++g_launches;
+  return cudaGetLastError() == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+}
+
+int augtree_replay_bwd(const augtree_plan_t *pl, const void *q_r, const void *k_r, const void *v_r, const void *k_p,
+                       const void *v_p, const void *o_r, const float *lse_r, const void *do_r, void *dq_r, void *dk_r,
+                       void *dv_r, float *dkp_acc, float *dvp_acc, void *ws, size_t ws_bytes, void *stream) {
+  int r = check_plan(pl);
+  if (r) return r;
+  if (!dkp_acc || !dvp_acc) return AUGTREE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (pl->flags & AUGTREE_FLAG_ZERO_PROMPT_GRAD) {
+    const size_t bytes = (size_t)pl->total_p * pl->h_kv * pl->head_dim * 4;
+    if (cudaMemsetAsync(dkp_acc, 0, bytes, st) != cudaSuccess || cudaMemsetAsync(dvp_acc, 0, bytes, st) != cudaSuccess)
+      return AUGTREE_ERR_CUDA;
+  }
+  if (pl->total_r == 0) return AUGTREE_OK;
+  if (!q_r || !k_r || !v_r || !k_p || !v_p || !o_r || !lse_r || !do_r || !dq_r || !dk_r || !dv_r) return AUGTREE_ERR_INVALID_ARG;
+  if (!aligned16(q_r) || !aligned16(k_r) || !aligned16(v_r) || !aligned16(k_p) || !aligned16(v_p) || !aligned16(o_r) ||
+      !aligned16(do_r) || !aligned16(dq_r) || !aligned16(dk_r) || !aligned16(dv_r) || !aligned16(dkp_acc) || !aligned16(dvp_acc))
+    return AUGTREE_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < pl->ws_bwd || !aligned16(ws)) return AUGTREE_ERR_WORKSPACE;
+  BwdArgs a;
+  a.q = q_r; a.d_o = do_r; a.o = o_r; a.lse = lse_r; a.q_tok = pl->total_r;
+  a.k0 = k_r; a.v0 = v_r; a.kv0_tok = pl->total_r; a.k1 = k_p; a.v1 = v_p; a.kv1_tok = pl->total_p;
+  a.dq = dq_r; a.dk_out = dk_r; a.dv_out = dv_r; a.dk_acc = dkp_acc; a.dv_acc = dvp_acc; a.causal_fp32 = 0;
+  a.d_segs = pl->d_seg_replay;
+  const Sched &s = pl->sched[SCHED_REPLAY_BWD];
+  return pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, st) : launch_bwd<64>(pl, s, a, ws, st);
+}
+
+int augtree_prefill_bwd(const augtree_plan_t *pl, const void *q_p, const void *k_p, const void *v_p, const void *o_p,
+                        const float *lse_p, const void *do_p, float *dkp_acc, float *dvp_acc, void *dq_p, void *dk_p,
+                        void *dv_p, void *ws, size_t ws_bytes, void *stream) {
+  int r = check_plan(pl);
+  if (r) return r;
+  if (!q_p || !k_p || !v_p || !o_p || !lse_p || !do_p || !dkp_acc || !dvp_acc || !dq_p) return AUGTREE_ERR_INVALID_ARG;
+  if (!aligned16(q_p) || !aligned16(k_p) || !aligned16(v_p) || !aligned16(o_p) || !aligned16(do_p) || !aligned16(dq_p) ||
+      !aligned16(dkp_acc) || !aligned16(dvp_acc) || !aligned16(dk_p) || !aligned16(dv_p))
+    return AUGTREE_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < pl->ws_bwd || !aligned16(ws)) return AUGTREE_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  BwdArgs a;
+  a.q = q_p; a.d_o = do_p; a.o = o_p; a.lse = lse_p; a.q_tok = pl->total_p;
+  a.k0 = k_p; a.v0 = v_p; a.kv0_tok = pl->total_p; a.k1 = k_p; a.v1 = v_p; a.kv1_tok = pl->total_p;
+  a.dq = dq_p; a.dk_out = nullptr; a.dv_out = nullptr; a.dk_acc = dkp_acc; a.dv_acc = dvp_acc; a.causal_fp32 = 1;
+  a.d_segs = pl->d_seg_prefill;
+  const Sched &s = pl->sched[SCHED_PREFILL_BWD];
+  r = pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, st) : launch_bwd<64>(pl, s, a, ws, st);
+  if (r) return r;
+  const long long n4 = pl->total_p * (long long)pl->h_kv * pl->head_dim / 4;
+  if (dk_p) { cast_bf16_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(dkp_acc, static_cast<__nv_bfloat16 *>(dk_p), n4); ++g_launches; }
+  if (dv_p) { cast_bf16_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(dvp_acc, static_cast<__nv_bfloat16 *>(dv_p), n4); ++g_launches; }
+  return cudaGetLastError() == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+}
+
+int augtree_last_device_status(const augtree_plan_t *pl, int *status, int *detail) {
+  int r = check_plan(pl);
+  if (r || !status) return AUGTREE_ERR_INVALID_ARG;
+  int prev = 0;
+  cudaGetDevice(&prev);
+  cudaSetDevice(pl->device);
+  int h[2] = {0, 0};
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(h, pl->d_status, sizeof(h), cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess && (h[0] || h[1])) e = cudaMemset(pl->d_status, 0, sizeof(h));
+  cudaSetDevice(prev);
+  if (e != cudaSuccess) return AUGTREE_ERR_CUDA;
+  *status = h[0];
+  if (detail) *detail = h[1];
+  return AUGTREE_OK;
+}
+
+long long augtree_launch_count(void) { return g_launches.load(); }
+
+const char *augtree_status_string(int s) {
+  switch (s) {
+    case AUGTREE_OK: return "ok";
+    case AUGTREE_ERR_INVALID_ARG: return "invalid argument";
+    case AUGTREE_ERR_UNSUPPORTED: return "unsupported configuration";
+    case AUGTREE_ERR_WORKSPACE: return "workspace missing or too small";
+    case AUGTREE_ERR_CUDA: return "CUDA call failed";
+    case AUGTREE_ERR_TIMEOUT: return "device-side wait timed out";
+    case AUGTREE_ERR_INTERNAL: return "internal error";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,208 @@
+// Pack & schedule (host): prefix sums, work items for the four kernels and their
+// largest-first assignment to replay lanes.
+//
+// Units and weights follow Sec. 3.4 ("Replay units and grid assignment"): a
+// unit's weight is its valid Q-KV tile count, and units are placed on lanes so
+// that the heaviest lane is as light as possible (Eq. 6 with one round), by
+// largest-first greedy balancing.  On one GPU a lane is a persistent CTA, so a
+// unit is one (query tile, head) for the forward kernels and one (KV tile, KV
+// head) for the backward kernels rather than a whole response path.
+//
+// Canonical item order (ids are positions in this order):
+//   prefill fwd : group, kv head, query tile, query head inside the kv head
+//   replay  fwd : group, kv head, branch, query tile, query head, prompt-KV shard
+//   replay  bwd : group, kv head, [prompt kv tiles, then branch by branch its kv tiles]
+//   prefill bwd : group, kv head, kv tile
+// Assignment: ids sorted by (weight descending, id ascending); each goes to the
+// lane with the smallest load so far (lowest lane index on ties).  Inside a
+// lane items run in ascending id, which keeps lanes on the same kv head at
+// about the same time so that the head's K/V stay in L2.
+#include "plan.h"
+
+#include <algorithm>
+#include <cmath>
+#include <numeric>
+#include <queue>
+
+namespace augtree {
+
+static inline int cdiv(int a, int b) { return (a + b - 1) / b; }
+
+static void assign_lanes(Sched &s, int weight_field, int n_lanes) {
+  const int n = s.n_items();
+  std::vector<int32_t> ids(n);
+  std::iota(ids.begin(), ids.end(), 0);
+  const int32_t *it = s.items.data();
+  const int ni = s.item_ints;
+  std::stable_sort(ids.begin(), ids.end(), [&](int32_t a, int32_t b) {
+    return it[(size_t)a * ni + weight_field] > it[(size_t)b * ni + weight_field];
+  });
+  typedef std::pair<int64_t, int32_t> LL;  // (load, lane): smallest load first, then lowest lane
+  std::priority_queue<LL, std::vector<LL>, std::greater<LL>> heap;
+  for (int l = 0; l < n_lanes; ++l) heap.push(LL(0, l));
+  std::vector<std::vector<int32_t>> per_lane(n_lanes);
+  for (int32_t id : ids) {
+    LL top = heap.top();
+    heap.pop();
+    per_lane[top.second].push_back(id);
+    heap.push(LL(top.first + it[(size_t)id * ni + weight_field], top.second));
+  }
+  s.lane_ptr.assign(n_lanes + 1, 0);
+  s.order.clear();
+  s.order.reserve(n);
+  for (int l = 0; l < n_lanes; ++l) {
+    std::sort(per_lane[l].begin(), per_lane[l].end());
+    s.order.insert(s.order.end(), per_lane[l].begin(), per_lane[l].end());
+    s.lane_ptr[l + 1] = (int32_t)s.order.size();
+  }
+}
+
+int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
+  if (!d || !p) return AUGTREE_ERR_INVALID_ARG;
+  if (d->struct_size != sizeof(augtree_desc_t) || d->version != AUGTREE_VERSION) return AUGTREE_ERR_INVALID_ARG;
+  if (d->n_groups < 1 || !d->prompt_len || !d->n_branches) return AUGTREE_ERR_INVALID_ARG;
+  if (d->h_q < 1 || d->h_kv < 1 || d->n_lanes < 0 || d->kv_splits < 0) return AUGTREE_ERR_INVALID_ARG;
+  if (d->h_q % d->h_kv != 0) return AUGTREE_ERR_UNSUPPORTED;
+  if (d->head_dim != 64 && d->head_dim != 128) return AUGTREE_ERR_UNSUPPORTED;
+  if (!(d->softmax_scale >= 0.f) || std::isinf(d->softmax_scale)) return AUGTREE_ERR_INVALID_ARG;
+
+  p->n_groups = d->n_groups;
+  p->h_q = d->h_q; p->h_kv = d->h_kv; p->head_dim = d->head_dim;
+  p->scale = d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / std::sqrt((float)d->head_dim);
+  p->flags = d->flags;
+  p->n_lanes = d->n_lanes;
+  p->kv_splits = d->kv_splits < 1 ? 1 : d->kv_splits;
+  if (p->kv_splits > 64) return AUGTREE_ERR_UNSUPPORTED;
+
+  p->prompt_len.assign(d->prompt_len, d->prompt_len + d->n_groups);
+  p->n_br.assign(d->n_branches, d->n_branches + d->n_groups);
+  int64_t nb = 0, tp = 0;
+  p->cu_p.assign(1, 0); p->cu_b.assign(1, 0);
+  for (int g = 0; g < d->n_groups; ++g) {
+    if (p->prompt_len[g] < 1 || p->n_br[g] < 0) return AUGTREE_ERR_INVALID_ARG;
+    tp += p->prompt_len[g]; nb += p->n_br[g];
+    if (tp > 0x3fffffff || nb > 0x3fffffff) return AUGTREE_ERR_UNSUPPORTED;
+    p->cu_p.push_back((int32_t)tp); p->cu_b.push_back((int32_t)nb);
+  }
+  if (nb > 0 && !d->branch_len) return AUGTREE_ERR_INVALID_ARG;
+  p->n_branches = (int32_t)nb;
+  p->branch_len.assign(d->branch_len, d->branch_len + nb);
+  int64_t tr = 0;
+  p->cu_r.assign(1, 0);
+  for (int64_t i = 0; i < nb; ++i) {
+    if (p->branch_len[i] < 1) return AUGTREE_ERR_INVALID_ARG;
+    tr += p->branch_len[i];
+    if (tr > 0x3fffffff) return AUGTREE_ERR_UNSUPPORTED;
+    p->cu_r.push_back((int32_t)tr);
+  }
+  p->total_p = tp; p->total_r = tr;
+  p->branch_group.resize(nb);
+  for (int g = 0; g < d->n_groups; ++g)
+    for (int i = p->cu_b[g]; i < p->cu_b[g + 1]; ++i) p->branch_group[i] = g;
+
+  const int rep = p->h_q / p->h_kv;
+  const int ng = p->n_groups;
+
+  // q-segment tables for the backward kernels
+  p->seg_replay.clear(); p->seg_prefill.clear();
+  for (int i = 0; i < (int)nb; ++i) { p->seg_replay.push_back(p->cu_r[i]); p->seg_replay.push_back(p->branch_len[i]); }
+  for (int g = 0; g < ng; ++g) { p->seg_prefill.push_back(p->cu_p[g]); p->seg_prefill.push_back(p->prompt_len[g]); }
+
+  // prompt-KV shards per group: shard = a run of whole KV tiles
+  p->group_splits.resize(ng);
+  std::vector<int> shard_tiles(ng);
+  p->max_splits = 1;
+  for (int g = 0; g < ng; ++g) {
+    const int na = cdiv(p->prompt_len[g], kTileKV);
+    const int want = std::min(p->kv_splits, na);
+    shard_tiles[g] = cdiv(na, want);
+    p->group_splits[g] = cdiv(na, shard_tiles[g]);
+    p->max_splits = std::max(p->max_splits, p->group_splits[g]);
+  }
+
+  Sched &pf = p->sched[SCHED_PREFILL_FWD], &rf = p->sched[SCHED_REPLAY_FWD];
+  Sched &rb = p->sched[SCHED_REPLAY_BWD], &pb = p->sched[SCHED_PREFILL_BWD];
+  pf.item_ints = rf.item_ints = AUGTREE_FWD_ITEM_INTS;
+  rb.item_ints = pb.item_ints = AUGTREE_BWD_ITEM_INTS;
+  pf.items.clear(); rf.items.clear(); rb.items.clear(); pb.items.clear();
+
+  for (int g = 0; g < ng; ++g) {
+    const int P = p->prompt_len[g], p0 = p->cu_p[g];
+    const int nqt_p = cdiv(P, kTileQ);
+    for (int c = 0; c < p->h_kv; ++c) {
+      // ---- prefill forward ----
+      for (int t = 0; t < nqt_p; ++t) {
+        const int rows = std::min(kTileQ, P - t * kTileQ);
+        const int blen = t * kTileQ + rows;
+        for (int j = 0; j < rep; ++j) {
+          const int32_t it[AUGTREE_FWD_ITEM_INTS] = {p0 + t * kTileQ, t * kTileQ, rows, c * rep + j, 0, 0, p0, blen,
+                                                     0, 1, cdiv(blen, kTileKV), c};
+          pf.items.insert(pf.items.end(), it, it + AUGTREE_FWD_ITEM_INTS);
+        }
+      }
+      // ---- replay forward ----
+      for (int b = p->cu_b[g]; b < p->cu_b[g + 1]; ++b) {
+        const int R = p->branch_len[b], r0 = p->cu_r[b];
+        const int ns = p->group_splits[g];
+        for (int t = 0; t < cdiv(R, kTileQ); ++t) {
+          const int rows = std::min(kTileQ, R - t * kTileQ);
+          const int blen = t * kTileQ + rows;
+          for (int j = 0; j < rep; ++j)
+            for (int s = 0; s < ns; ++s) {
+              const int a0 = s * shard_tiles[g] * kTileKV;
+              const int alen = std::min(P - a0, shard_tiles[g] * kTileKV);
+              const int bl = (s == ns - 1) ? blen : 0;
+              const int32_t it[AUGTREE_FWD_ITEM_INTS] = {r0 + t * kTileQ, t * kTileQ, rows, c * rep + j, p0 + a0, alen,
+                                                         r0, bl, s, ns, cdiv(alen, kTileKV) + cdiv(bl, kTileKV), c};
+              rf.items.insert(rf.items.end(), it, it + AUGTREE_FWD_ITEM_INTS);
+            }
+        }
+      }
+      // ---- replay backward: prompt kv tiles (mode 1), then each branch's kv tiles (mode 0) ----
+      const int b0 = p->cu_b[g], b1 = p->cu_b[g + 1];
+      if (b1 > b0) {
+        int visits = 0;
+        for (int b = b0; b < b1; ++b) visits += cdiv(p->branch_len[b], kTileQ) * rep;
+        for (int t = 0; t < cdiv(P, kTileKV); ++t) {
+          const int32_t it[AUGTREE_BWD_ITEM_INTS] = {p0 + t * kTileKV, t * kTileKV, std::min(kTileKV, P - t * kTileKV), c,
+                                                     1, b0, b1 - b0, visits};
+          rb.items.insert(rb.items.end(), it, it + AUGTREE_BWD_ITEM_INTS);
+        }
+      }
+      for (int b = b0; b < b1; ++b) {
+        const int R = p->branch_len[b], r0 = p->cu_r[b];
+        const int nt = cdiv(R, kTileKV);
+        for (int t = 0; t < nt; ++t) {
+          const int32_t it[AUGTREE_BWD_ITEM_INTS] = {r0 + t * kTileKV, t * kTileKV, std::min(kTileKV, R - t * kTileKV), c,
+                                                     0, b, 1, (cdiv(R, kTileQ) - t) * rep};
+          rb.items.insert(rb.items.end(), it, it + AUGTREE_BWD_ITEM_INTS);
+        }
+      }
+      // ---- prefill backward ----
+      for (int t = 0; t < cdiv(P, kTileKV); ++t) {
+        const int32_t it[AUGTREE_BWD_ITEM_INTS] = {p0 + t * kTileKV, t * kTileKV, std::min(kTileKV, P - t * kTileKV), c,
+                                                   0, g, 1, (nqt_p - t) * rep};
+        pb.items.insert(pb.items.end(), it, it + AUGTREE_BWD_ITEM_INTS);
+      }
+    }
+  }
+  if (p->n_lanes > 0) {
+    assign_lanes(pf, 10, p->n_lanes);
+    assign_lanes(rf, 10, p->n_lanes);
+    assign_lanes(rb, 7, p->n_lanes);
+    assign_lanes(pb, 7, p->n_lanes);
+  }
+
+  // scratch sizes (bytes, each region 256-byte aligned)
+  auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  const size_t hq = (size_t)p->h_q, dd = (size_t)p->head_dim;
+  p->ws_fwd = 0;
+  if (p->max_splits > 1)
+    p->ws_fwd = al((size_t)p->max_splits * (size_t)tr * hq * dd * 4) + al((size_t)p->max_splits * (size_t)tr * hq * 4);
+  const size_t tmax = (size_t)std::max<int64_t>(tp, tr);
+  // backward: dq accumulator fp32 [tokens,H_q,d], delta and scaled lse [H_q,tokens] fp32
+  p->ws_bwd = al(tmax * hq * dd * 4) + 2 * al(tmax * hq * 4);
+  return AUGTREE_OK;
+}
+
+}  // namespace augtree

@@ -1,0 +1,47 @@
+// Internal plan object: packing metadata on the host and its device copies.
+#pragma once
+#include <cstdint>
+#include <vector>
+
+#include "../../include/augtree.h"
+
+namespace augtree {
+
+constexpr int kTileQ = 128;   // query rows per tile
+constexpr int kTileKV = 128;  // keys per tile
+
+enum { SCHED_PREFILL_FWD = 0, SCHED_REPLAY_FWD = 1, SCHED_REPLAY_BWD = 2, SCHED_PREFILL_BWD = 3, SCHED_COUNT = 4 };
+
+struct Sched {
+  int item_ints = 0;
+  std::vector<int32_t> items;     // canonical order, item_ints per item
+  std::vector<int32_t> lane_ptr;  // [n_lanes + 1]
+  std::vector<int32_t> order;     // item ids, lane by lane
+  int32_t *d_items = nullptr;     // items gathered into lane order (device)
+  int32_t *d_lane_ptr = nullptr;  // (device)
+  int n_items() const { return item_ints ? (int)(items.size() / item_ints) : 0; }
+};
+
+}  // namespace augtree
+
+struct augtree_plan {
+  int32_t n_groups = 0, n_branches = 0;
+  int32_t h_q = 0, h_kv = 0, head_dim = 0;
+  float scale = 0.f;
+  uint32_t flags = 0;
+  int32_t n_lanes = 0, kv_splits = 1, max_splits = 1;
+  int device = -1;
+  int64_t total_p = 0, total_r = 0;
+  std::vector<int32_t> prompt_len, n_br, branch_len;
+  std::vector<int32_t> cu_p, cu_b, cu_r, branch_group, group_splits;
+  std::vector<int32_t> seg_replay, seg_prefill;
+  augtree::Sched sched[augtree::SCHED_COUNT];
+  int32_t *d_seg_replay = nullptr, *d_seg_prefill = nullptr, *d_branch_group = nullptr, *d_group_splits = nullptr;
+  int32_t *d_cu_r = nullptr;
+  int *d_status = nullptr;  // [2]: status, detail
+  size_t ws_fwd = 0, ws_bwd = 0;
+};
+
+namespace augtree {
+int build_plan_host(const augtree_desc_t *desc, augtree_plan *plan);
+}

@@ -1,0 +1,128 @@
+"""Host-side checks that need no GPU: the library loads, exports what the header
+declares, validates descriptors, and its packing tables equal the independent
+Python restatement bit for bit."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2609_33133_b200 import build
+    build.build()
+    from paper_2609_33133_b200 import binding as b
+    return b
+
+
+def test_exports_every_declared_symbol(binding):
+    header = open(os.path.join(ROOT, "include", "augtree.h")).read()
+    declared = set(re.findall(r"\b(augtree_[a-z_]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert hasattr(binding.lib, name), name
+
+
+def test_descriptor_validation(binding):
+    B = binding
+    with pytest.raises(B.AugtreeError) as e:
+        B.Plan([16], [[4]], 3, 2, 64, device=None, n_lanes=4)
+    assert e.value.code == -2                    # h_q % h_kv
+    with pytest.raises(B.AugtreeError) as e:
+        B.Plan([16], [[4]], 4, 2, 96, device=None, n_lanes=4)
+    assert e.value.code == -2                    # head_dim
+    with pytest.raises(B.AugtreeError) as e:
+        B.Plan([0], [[4]], 4, 2, 64, device=None, n_lanes=4)
+    assert e.value.code == -1                    # empty prompt
+    with pytest.raises(B.AugtreeError) as e:
+        B.Plan([16], [[4, 0]], 4, 2, 64, device=None, n_lanes=4)
+    assert e.value.code == -1                    # empty branch
+    with pytest.raises(B.AugtreeError) as e:
+        B.Plan([16], [[4]], 4, 2, 64, device=None, n_lanes=0)
+    assert e.value.code == -1                    # host-only plan needs a lane count
+    d = B.Desc(4, 1, 1, None, None, None, 4, 2, 64, 0.0, 0, 4, 0)   # wrong struct_size
+    h = C.c_void_p()
+    assert B.lib.augtree_plan_create(C.byref(d), -1, C.byref(h)) == -1
+    assert B.lib.augtree_plan_create(None, -1, C.byref(h)) == -1
+    assert B.lib.augtree_status_string(-5).decode().startswith("device-side wait")
+    # launches on a host-only plan are refused, not crashed
+    p = B.Plan([16], [[4]], 4, 2, 64, device=None, n_lanes=4)
+    assert B.lib.augtree_prefill_fwd(p._h, None, None, None, None, None, None, 0, None) == -1
+
+
+CASES = [
+    ([256], [[128] * 4], 4, 4, 148, 1),
+    ([300, 1, 129], [[5, 130, 257], [], [64]], 8, 2, 7, 1),
+    ([1000, 2000], [[100, 300], [50]], 4, 1, 16, 3),
+    ([8192], [[2048] * 8], 28, 4, 148, 1),
+]
+
+
+@pytest.mark.parametrize("pl,bl,hq,hkv,lanes,splits", CASES)
+def test_tables_bit_exact(binding, pl, bl, hq, hkv, lanes, splits):
+    from oracle import packing
+    B = binding
+    plan = B.Plan(pl, bl, hq, hkv, 128, device=None, n_lanes=lanes, kv_splits=splits)
+    ref = packing.build_tables(pl, bl, hq, hkv, splits)
+    assert (plan.metadata(B.TBL_CU_PROMPT) == ref["cu_p"]).all()
+    assert (plan.metadata(B.TBL_CU_BRANCH) == ref["cu_b"]).all()
+    assert (plan.metadata(B.TBL_CU_RESPONSE) == ref["cu_r"]).all()
+    assert (plan.metadata(B.TBL_GROUP_SPLITS) == ref["group_splits"]).all()
+    assert (plan.metadata(B.TBL_REPLAY_SEGMENTS).reshape(-1, 2) == ref["seg_replay"]).all()
+    assert (plan.metadata(B.TBL_PREFILL_SEGMENTS).reshape(-1, 2) == ref["seg_prefill"]).all()
+    for base, key, w, wf in [(B.TBL_PREFILL_FWD_ITEMS, "prefill_fwd", 12, 10), (B.TBL_REPLAY_FWD_ITEMS, "replay_fwd", 12, 10),
+                             (B.TBL_REPLAY_BWD_ITEMS, "replay_bwd", 8, 7), (B.TBL_PREFILL_BWD_ITEMS, "prefill_bwd", 8, 7)]:
+        items = plan.metadata(base).reshape(-1, w)
+        assert items.shape == ref[key].shape and (items == ref[key]).all(), key
+        ptr, order = packing.assign_lanes(ref[key][:, wf], lanes)
+        assert (plan.metadata(base + 1) == ptr).all(), key
+        assert (plan.metadata(base + 2) == order).all(), key
+        assert sorted(order.tolist()) == list(range(len(order)))
+
+
+def test_item_weights_count_visible_pairs():
+    """Forward items cover every visible (query, key) pair exactly once; backward items likewise."""
+    from oracle import packing, tree_attention as ora
+    pl, bl, hq, hkv = [300, 129], [[5, 130, 257], [64]], 4, 2
+    ref = packing.build_tables(pl, bl, hq, hkv, 2)
+    tb = ora.TreeBatch(pl, bl, hq, hkv, 128)
+    pre, rep, _ = ora.valid_pairs(tb)
+
+    def fwd_pairs(items):
+        tot = 0
+        for it in items:
+            q_pos0, rows, a_len, b_len = int(it[1]), int(it[2]), int(it[5]), int(it[7])
+            tot += rows * a_len
+            if b_len:
+                tot += sum(q_pos0 + r + 1 for r in range(rows))
+        return tot
+    assert fwd_pairs(ref["prefill_fwd"]) == pre * hq
+    assert fwd_pairs(ref["replay_fwd"]) == rep * hq
+
+    def bwd_pairs(items, segs):
+        tot = 0
+        for it in items:
+            kv_pos0, kv_rows, mode, seg0, nseg = int(it[1]), int(it[2]), int(it[4]), int(it[5]), int(it[6])
+            for s in range(seg0, seg0 + nseg):
+                L = int(segs[s][1])
+                for k in range(kv_pos0, kv_pos0 + kv_rows):
+                    tot += L if mode else max(0, L - k)
+        return tot * (hq // hkv)
+    assert bwd_pairs(ref["prefill_bwd"], ref["seg_prefill"]) == pre * hq
+    assert bwd_pairs(ref["replay_bwd"], ref["seg_replay"]) == rep * hq
+
+
+def test_greedy_assignment_within_lpt_bound():
+    from oracle import packing
+    rng = np.random.default_rng(0)
+    for _ in range(20):
+        n, m = int(rng.integers(3, 10)), int(rng.integers(2, 4))
+        w = [int(x) for x in rng.integers(1, 30, n)]
+        ptr, order = packing.assign_lanes(w, m)
+        got = packing.makespan(w, ptr, order)
+        opt = packing.brute_force_makespan(w, m)
+        assert opt <= got <= opt * (4 / 3 - 1 / (3 * m)) + 1e-9
