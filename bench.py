@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Benchmark of the tree-attention hot path (prefill + replay, forward + backward) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--config I]
+
+One "step" is one pass of the whole path over one batch of synthetic groups:
+augtree_prefill_fwd -> augtree_replay_fwd -> augtree_replay_bwd -> augtree_prefill_bwd.
+At N = 1 the workload is the 7B-shaped layer (configuration 2).  With N > 1 every
+rank runs its own group of the same shape (independent trees shard with no
+exchange step), so the scaling is weak and there is no data-path collective.
+
+Prints one JSON line (rank 0).  `value` is useful TFLOP/s: causal-masked pairs
+only, the prompt counted once, 14 * d FLOP per (query, key) pair and query head.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+from paper_2609_33133_b200 import workloads as wl  # noqa: E402
+
+METRIC = "tree-attn fwd+bwd useful TFLOP/s (speedup vs flattened in 'flattened')"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
+def tri(n):
+    return n * (n + 1) // 2
+
+
+def pair_counts(w):
+    pre = sum(tri(p) for p in w.prompt_len)
+    rep = sum(r * p + tri(r) for p, bl in zip(w.prompt_len, w.branch_len) for r in bl)
+    flat = sum(tri(p + r) for p, bl in zip(w.prompt_len, w.branch_len) for r in (bl if bl else [0]))
+    return pre, rep, flat
+
+
+def useful_flops(w):
+    pre, rep, flat = pair_counts(w)
+    per_pair = 14 * w.head_dim * w.h_q
+    return {"total": per_pair * (pre + rep), "prefill_fwd": 4 * w.head_dim * w.h_q * pre, "replay_fwd": 4 * w.head_dim * w.h_q * rep,
+            "replay_bwd": 10 * w.head_dim * w.h_q * rep, "prefill_bwd": 10 * w.head_dim * w.h_q * pre,
+            "flattened_total": per_pair * flat, "reuse_factor": flat / (pre + rep)}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"bf16_tflops": float(p["bf16_tflops"]), "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"bf16_tflops": FALLBACK_BF16_TFLOPS, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(pw), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- #
+def oracle_sample(w, seconds_budget=20.0):
+    """Times the fp64 oracle, as it stands, on whole (branch, query head) flattened
+    sequences of the workload until the budget is used, and extrapolates to all of them."""
+    from oracle import tree_attention as ora
+    g = 0
+    P, bl = w.prompt_len[g], w.branch_len[g]
+    # tensors of group 0, one KV head and its first query head are enough for the sample
+    gen = torch.Generator().manual_seed(w.seed)
+    n_seq_total = sum(len(b) if b else 1 for b in w.branch_len) * w.h_q
+    done, t_used, flops_flat = 0, 0.0, 0
+    cores = len(os.sched_getaffinity(0))
+    for r in (bl if bl else [0]):
+        n = P + r
+        q, k, v, do = (torch.randn((n, w.head_dim), generator=gen).to(torch.bfloat16).double().numpy() for _ in range(4))
+        t0 = time.perf_counter()
+        o, lse, p = ora.causal_attention_fwd(q, k, v, 1.0 / np.sqrt(w.head_dim))
+        ora.causal_attention_bwd(q, k, v, o, p, do, 1.0 / np.sqrt(w.head_dim))
+        t_used += time.perf_counter() - t0
+        done += 1
+        flops_flat += 14 * w.head_dim * tri(n)
+        if t_used > seconds_budget:
+            break
+    # the sampled sequences stand for all (branch, head) sequences of the same group shape
+    est_total_s = t_used / done * n_seq_total
+    return {"seconds_sample": t_used, "sequences": done, "of": n_seq_total, "est_total_s": est_total_s, "cores": cores}
+
+
+def run_reference(args, w):
+    """--impl reference: the fp64 CPU oracle on a bounded sample per step."""
+    fl = useful_flops(w)
+    times = []
+    info = None
+    for i in range(args.warmup + args.steps):
+        info = oracle_sample(w, seconds_budget=8.0)
+        if i >= args.warmup:
+            times.append(info["est_total_s"])
+    est = statistics.mean(times)
+    val = fl["total"] / est / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": {"workload": w.name, "tokens": w.total_prompt + w.total_response},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": info["cores"], "kind": "oracle",
+                             "sample": f"{info['sequences']} of {info['of']} flattened (branch, head) sequences per step, time extrapolated"},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- #
+def time_steps(step_fn, steps, warmup, dist, sampler_index=None):
+    """W warm-up steps, then K steps between two events, bracketed by barrier + synchronize; max over ranks."""
+    for _ in range(warmup):
+        step_fn()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(sampler_index) if sampler_index is not None else None
+    if sampler:
+        sampler.__enter__()
+        time.sleep(0.15)
+    e0.record()
+    for _ in range(steps):
+        step_fn()
+    e1.record()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.__exit__()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms, (sampler.summary() if sampler else None)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="workload configuration 1..5 (default 2, the metric's)")
+    ap.add_argument("--no-flattened", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    w = wl.config(args.config)
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, w)
+        return 0
+
+    from paper_2609_33133_b200 import build
+    build.build()
+    from paper_2609_33133_b200 import binding as B
+
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist = dist_mod
+    w.seed += rank  # every rank replays its own trees of the same shape
+    fl = useful_flops(w)
+    pk = peaks()
+
+    big = (w.total_prompt + w.total_response) * w.h_q * w.head_dim > 2e8
+    t_dev = wl.make_tensors(w, device="cuda" if big else "cpu")
+    t_dev = {k: v.cuda() for k, v in t_dev.items()}
+    splits = 4 if w.extra.get("force_split") else 0
+    plan = B.Plan(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, device=local_rank, flags=B.FLAG_ZERO_PROMPT_GRAD,
+                  kv_splits=splits)
+    out = B.alloc_outputs(plan)
+
+    def step():
+        B.run_forward_backward(plan, t_dev, out)
+
+    # ---- main timed region (inputs resident in HBM), with per-kernel events for the roofline
+    plan.set_timing(True)
+    l0 = B.launch_count()
+    ms, clocks = time_steps(step, args.steps, args.warmup, dist, sampler_index=local_rank if rank == 0 else None)
+    launches = (B.launch_count() - l0) // (args.steps + args.warmup) * args.steps
+    st = plan.device_status()
+    if st != (0, 0):
+        raise RuntimeError(f"device status {st}")
+    kt = [plan.kernel_time(k) for k in range(4)]
+    plan.set_timing(False)
+    ms_step = ms / args.steps
+    value = world * fl["total"] / (ms_step * 1e-3) / 1e12
+
+    # dominant kernel: the replay backward tile kernel
+    names = ["prefill_fwd", "replay_fwd", "replay_bwd", "prefill_bwd"]
+    per_kernel = {}
+    for n, (tot, cnt) in zip(names, kt):
+        if cnt:
+            per_kernel[n] = {"ms": tot / cnt, "tflops": fl[n] / (tot / cnt * 1e-3) / 1e12, "launches": cnt}
+    dom = max(per_kernel, key=lambda n: per_kernel[n]["ms"])
+    roofline = {"bound": "tensor", "kernel": f"{'bwd' if 'bwd' in dom else 'fwd'}_kernel ({dom})", "achieved": per_kernel[dom]["tflops"],
+                "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": per_kernel[dom]["tflops"] / pk["bf16_tflops"],
+                "peak_source": f"{pk['source']} cuBLAS bf16 burst", "traffic": None}
+
+    # ---- end to end: pinned host inputs copied in, results copied out, every step
+    host_in = {k: v.cpu().pin_memory() for k, v in t_dev.items()}
+    res_names = ["o_p", "lse_p", "o_r", "lse_r", "dq_p", "dq_r", "dk_r", "dv_r", "dk_p", "dv_p"]
+    host_out = {k: torch.empty(out[k].shape, dtype=out[k].dtype).pin_memory() for k in res_names}
+    h2d = sum(v.numel() * v.element_size() for v in host_in.values())
+    d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+
+    def step_e2e():
+        for k, v in host_in.items():
+            t_dev[k].copy_(v, non_blocking=True)
+        B.run_forward_backward(plan, t_dev, out)
+        for k, v in host_out.items():
+            v.copy_(out[k], non_blocking=True)
+
+    ms_e2e, _ = time_steps(step_e2e, max(3, args.steps // 2), 3, dist)
+    ms_e2e /= max(3, args.steps // 2)
+    e2e = {"value": world * fl["total"] / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    # ---- flattened no-reuse baseline: same kernels, prompt duplicated per branch
+    flat = None
+    if not args.no_flattened and rank == 0:
+        del host_in, host_out
+        fw = w.flattened()
+        ft = wl.flatten_tensors(w, {k: v for k, v in t_dev.items()})
+        e = lambda h: torch.empty((0, h, w.head_dim), dtype=torch.bfloat16, device="cuda")
+        ft.update({"q_r": e(w.h_q), "k_r": e(w.h_kv), "v_r": e(w.h_kv), "do_r": e(w.h_q)})
+        fplan = B.Plan(fw.prompt_len, fw.branch_len, fw.h_q, fw.h_kv, fw.head_dim, device=local_rank, flags=B.FLAG_ZERO_PROMPT_GRAD)
+        fout = B.alloc_outputs(fplan)
+        fsteps = max(3, args.steps // 4)
+        fms, _ = time_steps(lambda: B.run_forward_backward(fplan, ft, fout), fsteps, 3, None)
+        fms /= fsteps
+        flat = {"ms_per_step": fms, "speedup": fms / ms_step, "reuse_factor": fl["reuse_factor"],
+                "tflops_executed": fl["flattened_total"] / (fms * 1e-3) / 1e12}
+        del fout, ft
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        info = oracle_sample(w, seconds_budget=15.0)
+        cpu = {"value": fl["total"] / info["est_total_s"] / 1e12, "unit": "TFLOP/s", "cores": info["cores"], "kind": "oracle",
+               "sample": f"{info['sequences']} of {info['of']} flattened (branch, head) sequences, {info['seconds_sample']:.1f} s, extrapolated"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": w.name, "groups": w.n_groups, "prompt_tokens": w.total_prompt, "response_tokens": w.total_response,
+                       "h_q": w.h_q, "h_kv": w.h_kv, "head_dim": w.head_dim, "useful_tflop_per_step": fl["total"] / 1e12,
+                       "l2": "no flush: inputs + outputs exceed the 126 MB L2 (K/V reuse from L2 is part of the method)",
+                       "parallelism": f"independent groups x{world}"},
+            "pct_of_measured_bf16_peak": 100 * value / world / pk["bf16_tflops"],
+            "pct_of_nominal_bf16_peak": 100 * value / world / NOMINAL_BF16_TFLOPS,
+            "kernels": per_kernel, "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "flattened": flat, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -187,6 +187,20 @@ int augtree_prefill_bwd(const augtree_plan_t *plan, const void *q_p, const void 
  */
 int augtree_last_device_status(const augtree_plan_t *plan, int *status, int *detail);
 
+/*
+ * Measurement aid (no counterpart in the paper's method; Sec. 4.1 reports such
+ * per-kernel attention times).  With enable != 0 every later launch of the four
+ * tile kernels on this plan is bracketed by a pair of CUDA events recorded on
+ * the launch's stream (up to 512 launches per kernel, then recording stops);
+ * each call resets the record.  The events are created on the first call,
+ * which is therefore not free; the launches themselves stay asynchronous.
+ * augtree_get_kernel_time waits for the recorded launches of one kernel
+ * (0 prefill fwd, 1 replay fwd, 2 replay bwd, 3 prefill bwd) and returns their
+ * summed device time and count.
+ */
+int augtree_set_timing(augtree_plan_t *plan, int enable);
+int augtree_get_kernel_time(const augtree_plan_t *plan, int kernel, float *total_ms, int *launches);
+
 /* Number of kernel launches the library has enqueued since it was loaded. */
 long long augtree_launch_count(void);
 

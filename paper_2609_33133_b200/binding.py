@@ -28,7 +28,8 @@ FWD_ITEM_INTS, BWD_ITEM_INTS = 12, 8
 
 EXPORTS = ["augtree_plan_create", "augtree_plan_destroy", "augtree_plan_workspace_bytes", "augtree_plan_metadata",
            "augtree_prefill_fwd", "augtree_replay_fwd", "augtree_replay_bwd", "augtree_prefill_bwd",
-           "augtree_last_device_status", "augtree_launch_count", "augtree_status_string"]
+           "augtree_last_device_status", "augtree_launch_count", "augtree_status_string",
+           "augtree_set_timing", "augtree_get_kernel_time"]
 
 
 class Desc(C.Structure):
@@ -49,6 +50,8 @@ lib.augtree_replay_fwd.argtypes = [_vp] + [_vp] * 7 + [_vp, _sz, _vp]
 lib.augtree_replay_bwd.argtypes = [_vp] + [_vp] * 13 + [_vp, _sz, _vp]
 lib.augtree_prefill_bwd.argtypes = [_vp] + [_vp] * 11 + [_vp, _sz, _vp]
 lib.augtree_last_device_status.argtypes = [_vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+lib.augtree_set_timing.argtypes = [_vp, C.c_int]
+lib.augtree_get_kernel_time.argtypes = [_vp, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_int)]
 lib.augtree_launch_count.restype = C.c_longlong
 lib.augtree_status_string.restype = C.c_char_p
 lib.augtree_status_string.argtypes = [C.c_int]
@@ -99,7 +102,7 @@ class Plan:
 
     def __del__(self):
         h = getattr(self, "_h", None)
-        if h is not None and h.value:
+        if h is not None and h.value and lib is not None:
             lib.augtree_plan_destroy(h)
             self._h = None
 
@@ -132,6 +135,14 @@ class Plan:
         _check(lib.augtree_prefill_bwd(self._h, _ptr(q_p), _ptr(k_p), _ptr(v_p), _ptr(o_p), _ptr(lse_p), _ptr(do_p),
                                        _ptr(dkp_acc), _ptr(dvp_acc), _ptr(dq_p), _ptr(dk_p), _ptr(dv_p), _ptr(ws),
                                        0 if ws is None else ws.numel() * ws.element_size(), self._stream()), "prefill_bwd")
+
+    def set_timing(self, enable: bool):
+        _check(lib.augtree_set_timing(self._h, int(enable)), "set_timing")
+
+    def kernel_time(self, kernel: int):
+        ms, n = C.c_float(), C.c_int()
+        _check(lib.augtree_get_kernel_time(self._h, kernel, C.byref(ms), C.byref(n)), "get_kernel_time")
+        return ms.value, n.value
 
     def device_status(self):
         s, d = C.c_int(), C.c_int()

@@ -73,6 +73,8 @@ int upload_sched(Sched &s, int n_lanes) {
   return upload(s.lane_ptr, &s.d_lane_ptr);
 }
 
+void timing_mark(const augtree_plan *pl, int kind, bool stop, cudaStream_t st);
+
 template <int D>
 int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long q_tok, const void *ka, const void *va,
                long long a_tok, const void *kb, const void *vb, long long b_tok, void *o, float *lse, float *part_o,
@@ -95,7 +97,10 @@ int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long 
       return AUGTREE_ERR_CUDA;
     attr_set[D / 128] = true;
   }
+  const int kind = (int)(&s - pl->sched);
+  timing_mark(pl, kind, false, st);
   fwd_kernel<D><<<pl->n_lanes, kFwdThreads, FwdSmem<D>::kBytes, st>>>(mq, mka, mva, mkb, mvb, p);
+  timing_mark(pl, kind, true, st);
   ++g_launches;
   return cudaGetLastError() == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
 }
@@ -154,7 +159,10 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
         return AUGTREE_ERR_CUDA;
       attr_set[D / 128] = true;
     }
+    const int kind = (int)(&s - pl->sched);
+    timing_mark(pl, kind, false, st);
     bwd_kernel<D><<<pl->n_lanes, kBwdThreads, BwdSmem<D>::kBytes, st>>>(mq, mdo, mk0, mv0, mk1, mv1, p);
+    timing_mark(pl, kind, true, st);
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return AUGTREE_ERR_CUDA;
   }
@@ -164,6 +172,18 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     ++g_launches;
   }
   return cudaGetLastError() == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+}
+
+constexpr size_t kTimingPairs = 512;
+
+void timing_mark(const augtree_plan *pl, int kind, bool stop, cudaStream_t st) {
+  Timing *t = pl->timing;
+  if (!t || !t->on) return;
+  size_t &u = t->used[kind];
+  if (!stop && u + 2 > t->ev[kind].size()) return;  // pool exhausted: stop recording
+  if (stop && (u & 1) == 0) return;
+  cudaEventRecord(static_cast<cudaEvent_t>(t->ev[kind][u]), st);
+  ++u;
 }
 
 int check_plan(const augtree_plan *pl) {
@@ -229,6 +249,11 @@ int augtree_plan_destroy(augtree_plan_t *pl) {
     for (int k = 0; k < SCHED_COUNT; ++k) { cudaFree(pl->sched[k].d_items); cudaFree(pl->sched[k].d_lane_ptr); }
     cudaFree(pl->d_seg_replay); cudaFree(pl->d_seg_prefill); cudaFree(pl->d_branch_group); cudaFree(pl->d_group_splits);
     cudaFree(pl->d_cu_r); cudaFree(pl->d_status);
+    if (pl->timing) {
+      for (int k = 0; k < SCHED_COUNT; ++k)
+        for (void *e : pl->timing->ev[k]) cudaEventDestroy(static_cast<cudaEvent_t>(e));
+      delete pl->timing;
+    }
     cudaSetDevice(prev);
   }
   delete pl;
@@ -384,6 +409,45 @@ int augtree_last_device_status(const augtree_plan_t *pl, int *status, int *detai
   if (e != cudaSuccess) return AUGTREE_ERR_CUDA;
   *status = h[0];
   if (detail) *detail = h[1];
+  return AUGTREE_OK;
+}
+
+int augtree_set_timing(augtree_plan_t *pl, int enable) {
+  int r = check_plan(pl);
+  if (r) return r;
+  int prev = 0;
+  cudaGetDevice(&prev);
+  cudaSetDevice(pl->device);
+  if (!pl->timing) {
+    pl->timing = new (std::nothrow) Timing();
+    if (!pl->timing) { cudaSetDevice(prev); return AUGTREE_ERR_INTERNAL; }
+    for (int k = 0; k < SCHED_COUNT && !r; ++k)
+      for (size_t i = 0; i < 2 * kTimingPairs; ++i) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) { r = AUGTREE_ERR_CUDA; break; }
+        pl->timing->ev[k].push_back(e);
+      }
+  }
+  pl->timing->on = enable != 0 && !r;
+  for (int k = 0; k < SCHED_COUNT; ++k) pl->timing->used[k] = 0;
+  cudaSetDevice(prev);
+  return r;
+}
+
+int augtree_get_kernel_time(const augtree_plan_t *pl, int kernel, float *total_ms, int *launches) {
+  int r = check_plan(pl);
+  if (r || kernel < 0 || kernel >= SCHED_COUNT || !total_ms || !launches) return AUGTREE_ERR_INVALID_ARG;
+  *total_ms = 0.f; *launches = 0;
+  const Timing *t = pl->timing;
+  if (!t) return AUGTREE_OK;
+  for (size_t i = 0; i + 1 < t->used[kernel]; i += 2) {
+    cudaEvent_t a = static_cast<cudaEvent_t>(t->ev[kernel][i]), b = static_cast<cudaEvent_t>(t->ev[kernel][i + 1]);
+    if (cudaEventSynchronize(b) != cudaSuccess) return AUGTREE_ERR_CUDA;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, a, b) != cudaSuccess) return AUGTREE_ERR_CUDA;
+    *total_ms += ms;
+    ++*launches;
+  }
   return AUGTREE_OK;
 }
 

@@ -22,6 +22,13 @@ struct Sched {
   int n_items() const { return item_ints ? (int)(items.size() / item_ints) : 0; }
 };
 
+// CUDA-event pairs recorded around the tile kernels when timing is switched on.
+struct Timing {
+  bool on = false;
+  std::vector<void *> ev[SCHED_COUNT];  // cudaEvent_t start/stop pairs, in launch order
+  size_t used[SCHED_COUNT] = {0, 0, 0, 0};
+};
+
 }  // namespace augtree
 
 struct augtree_plan {
@@ -39,6 +46,7 @@ struct augtree_plan {
   int32_t *d_seg_replay = nullptr, *d_seg_prefill = nullptr, *d_branch_group = nullptr, *d_group_splits = nullptr;
   int32_t *d_cu_r = nullptr;
   int *d_status = nullptr;  // [2]: status, detail
+  augtree::Timing *timing = nullptr;  // optional CUDA-event timing of the tile kernels
   size_t ws_fwd = 0, ws_bwd = 0;
 };
 

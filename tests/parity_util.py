@@ -1,0 +1,54 @@
+"""Shared helpers of the GPU parity tests: run the CUDA path and the fp64 oracle on the same inputs."""
+import numpy as np
+import torch
+
+from oracle import tree_attention as ora
+from paper_2609_33133_b200 import workloads as wl
+
+REL_L2, MAX_ABS, LSE_ABS = 5e-3, 2e-2, 1e-3   # tolerances of the benchmark contract, against fp64
+GRADS = ["dq_p", "dk_p", "dv_p", "dq_r", "dk_r", "dv_r"]
+
+
+def run_gpu(B, w, t_cpu, kv_splits=0, n_lanes=0, flags=0):
+    plan = B.Plan(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, device=0, kv_splits=kv_splits,
+                  n_lanes=n_lanes, flags=flags)
+    t = {k: v.cuda() for k, v in t_cpu.items()}
+    out = B.alloc_outputs(plan)
+    B.run_forward_backward(plan, t, out)
+    torch.cuda.synchronize()
+    status = plan.device_status()
+    assert status == (0, 0), f"device status {status}"
+    return {k: v.float().cpu().numpy().astype(np.float64) for k, v in out.items() if k != "ws"}, plan
+
+
+def run_oracle(w, t_cpu):
+    tb = ora.TreeBatch(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim)
+    f = lambda x: x.float().numpy().astype(np.float64)
+    return ora.tree_attention_fwd_bwd(tb, *[f(t_cpu[n]) for n in wl.TENSOR_NAMES])
+
+
+def errors(got, ref):
+    rows = {}
+    for k in ref:
+        if ref[k].size == 0:
+            continue
+        diff = got[k] - ref[k]
+        finite = np.isfinite(got[k]).all()
+        denom = np.linalg.norm(ref[k].ravel())
+        rows[k] = (float(np.linalg.norm(diff.ravel()) / denom) if denom > 0 else 0.0, float(np.abs(diff).max()), bool(finite))
+    return rows
+
+
+def assert_parity(got, ref):
+    rows = errors(got, ref)
+    bad = []
+    for k, (rel, mx, finite) in rows.items():
+        if not finite:
+            bad.append((k, "non-finite"))
+        elif k.startswith("lse"):
+            if mx > LSE_ABS:
+                bad.append((k, rel, mx))
+        elif rel > REL_L2 or mx > MAX_ABS:
+            bad.append((k, rel, mx))
+    assert not bad, f"parity failures: {bad}; all: {rows}"
+    return rows
