@@ -200,6 +200,7 @@ def main():
     ap.add_argument("--config", type=int, default=2, help="workload configuration 1..5 (default 2, the metric's)")
     ap.add_argument("--no-flattened", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -276,10 +277,12 @@ def main():
         for k, v in host_out.items():
             v.copy_(out[k], non_blocking=True)
 
-    ms_e2e, _ = time_steps(step_e2e, max(3, args.steps // 2), 3, dist)
-    ms_e2e /= max(3, args.steps // 2)
-    e2e = {"value": world * fl["total"] / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
-           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    e2e = None
+    if not args.no_e2e:
+        ms_e2e, _ = time_steps(step_e2e, max(3, args.steps // 2), 3, dist)
+        ms_e2e /= max(3, args.steps // 2)
+        e2e = {"value": world * fl["total"] / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     # ---- flattened no-reuse baseline: same kernels, prompt duplicated per branch
     flat = None
