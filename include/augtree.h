@@ -181,6 +181,43 @@ int augtree_prefill_bwd(const augtree_plan_t *plan, const void *q_p, const void 
                         void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * augtree_replay_fwd for callers that cannot hand the library a scratch
+ * buffer.  (The paper has no counterpart: this is a packaging variant of the
+ * sharded replay forward, not a step of the method.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- a
+ * plug-in inside a host runtime that owns the allocator and only passes in
+ * pre-existing tensors, a real-time loop that must not take the allocator
+ * lock, a process whose memory is fully pre-partitioned.  Such a caller can
+ * point at its inputs and outputs but cannot obtain the `ws` block that the
+ * sharded forward needs for the per-shard partial softmax states.
+ *
+ * Here that scratch is a fixed array inside the library's device image,
+ * AUGTREE_STATIC_SCRATCH_BYTES (32 MiB) large.  Every GPU on which the
+ * library's code is loaded keeps those 32 MiB reserved until the process
+ * exits, whether or not this function is ever called.  The call performs no
+ * cudaMalloc / cudaFree and uses no allocating library routine; the plan must
+ * already exist (augtree_plan_create is the allocating step and belongs to
+ * set-up).
+ *
+ *  - A plan whose forward scratch need (augtree_plan_workspace_bytes, fwd)
+ *    exceeds the array is refused with AUGTREE_ERR_WORKSPACE; nothing is
+ *    launched.  Plans without prompt-KV shards need no scratch and always fit.
+ *  - The first call on each device looks up the array's device address (a
+ *    one-off set-up step, done with that device current).  Make that first
+ *    call outside any stream capture.
+ *  - All calls on a device share the one array and it keeps whatever the last
+ *    call left there.  Nothing in it has to start at zero: every value the
+ *    merge kernel reads is written by the same call's tile kernel first.  Two
+ *    calls that may overlap on the GPU (different streams, no dependency) race
+ *    on it; order them.
+ * Arguments and results are those of augtree_replay_fwd.
+ */
+#define AUGTREE_STATIC_SCRATCH_BYTES (32u << 20)
+int augtree_replay_fwd_static(const augtree_plan_t *plan, const void *q_r, const void *k_r, const void *v_r,
+                              const void *k_p, const void *v_p, void *o_r, float *lse_r, void *stream);
+
+/*
  * Synchronises the plan's device and reads the device status word: *status is
  * AUGTREE_OK or AUGTREE_ERR_TIMEOUT; *detail (may be NULL) gets a code that
  * names the wait that gave up.  The word is cleared by the read.

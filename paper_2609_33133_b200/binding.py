@@ -20,6 +20,7 @@ if not os.path.exists(LIB_PATH):
 lib = C.CDLL(LIB_PATH)
 
 FLAG_ZERO_PROMPT_GRAD = 1
+STATIC_SCRATCH_BYTES = 32 << 20
 FWD_ITEM_INTS, BWD_ITEM_INTS = 12, 8
 (TBL_CU_PROMPT, TBL_CU_BRANCH, TBL_CU_RESPONSE, TBL_PREFILL_FWD_ITEMS, TBL_PREFILL_FWD_LANE_PTR, TBL_PREFILL_FWD_ORDER,
  TBL_REPLAY_FWD_ITEMS, TBL_REPLAY_FWD_LANE_PTR, TBL_REPLAY_FWD_ORDER, TBL_REPLAY_BWD_ITEMS, TBL_REPLAY_BWD_LANE_PTR,
@@ -29,7 +30,7 @@ FWD_ITEM_INTS, BWD_ITEM_INTS = 12, 8
 EXPORTS = ["augtree_plan_create", "augtree_plan_destroy", "augtree_plan_workspace_bytes", "augtree_plan_metadata",
            "augtree_prefill_fwd", "augtree_replay_fwd", "augtree_replay_bwd", "augtree_prefill_bwd",
            "augtree_last_device_status", "augtree_launch_count", "augtree_status_string",
-           "augtree_set_timing", "augtree_get_kernel_time"]
+           "augtree_set_timing", "augtree_get_kernel_time", "augtree_replay_fwd_static"]
 
 
 class Desc(C.Structure):
@@ -47,6 +48,7 @@ lib.augtree_plan_workspace_bytes.argtypes = [_vp, C.POINTER(_sz), C.POINTER(_sz)
 lib.augtree_plan_metadata.argtypes = [_vp, C.c_int, _vp, C.POINTER(_sz)]
 lib.augtree_prefill_fwd.argtypes = [_vp] + [_vp] * 5 + [_vp, _sz, _vp]
 lib.augtree_replay_fwd.argtypes = [_vp] + [_vp] * 7 + [_vp, _sz, _vp]
+lib.augtree_replay_fwd_static.argtypes = [_vp] + [_vp] * 7 + [_vp]
 lib.augtree_replay_bwd.argtypes = [_vp] + [_vp] * 13 + [_vp, _sz, _vp]
 lib.augtree_prefill_bwd.argtypes = [_vp] + [_vp] * 11 + [_vp, _sz, _vp]
 lib.augtree_last_device_status.argtypes = [_vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
@@ -125,6 +127,12 @@ class Plan:
         _check(lib.augtree_replay_fwd(self._h, _ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(k_p), _ptr(v_p), _ptr(o_r),
                                       _ptr(lse_r), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
                                       self._stream()), "replay_fwd")
+
+    def replay_fwd_static(self, q_r, k_r, v_r, k_p, v_p, o_r, lse_r):
+        """replay_fwd with the shard scratch taken from the library's built-in 32 MiB device array:
+        for callers that cannot allocate a workspace.  Calls on one device share that array."""
+        _check(lib.augtree_replay_fwd_static(self._h, _ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(k_p), _ptr(v_p), _ptr(o_r),
+                                             _ptr(lse_r), self._stream()), "replay_fwd_static")
 
     def replay_bwd(self, q_r, k_r, v_r, k_p, v_p, o_r, lse_r, do_r, dq_r, dk_r, dv_r, dkp_acc, dvp_acc, ws):
         _check(lib.augtree_replay_bwd(self._h, _ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(k_p), _ptr(v_p), _ptr(o_r),

@@ -13,7 +13,15 @@
 
 using namespace augtree;
 
+// Built-in scratch of augtree_replay_fwd_static: part of the device image, so
+// each GPU that loads this library holds it until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[AUGTREE_STATIC_SCRATCH_BYTES];
+
 namespace {
+
+constexpr int kMaxStaticDevices = 64;
+void *g_static_ptr[kMaxStaticDevices] = {};  // device address of g_static_scratch, per device
+std::mutex g_static_mutex;
 
 std::atomic<long long> g_launches{0};
 
@@ -341,6 +349,34 @@ int augtree_replay_fwd(const augtree_plan_t *pl, const void *q_r, const void *k_
                                                pl->n_branches, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q);
   ++g_launches;
   return cudaGetLastError() == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+}
+
+// Replay forward without caller scratch: the shard partials live in
+// g_static_scratch (file scope, above).  In host code the array's name is only a
+// host-side handle, so its device address is looked up once per device, with
+// that device current, and handed to the ordinary entry point as its workspace.
+int augtree_replay_fwd_static(const augtree_plan_t *pl, const void *q_r, const void *k_r, const void *v_r,
+                              const void *k_p, const void *v_p, void *o_r, float *lse_r, void *stream) {
+  int r = check_plan(pl);
+  if (r) return r;
+  if (pl->ws_fwd > (size_t)AUGTREE_STATIC_SCRATCH_BYTES) return AUGTREE_ERR_WORKSPACE;  // need exceeds the built-in array
+  if (pl->device >= kMaxStaticDevices) return AUGTREE_ERR_UNSUPPORTED;
+  void *scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[pl->device]) {
+      int cur = -1;
+      if (cudaGetDevice(&cur) != cudaSuccess) return AUGTREE_ERR_CUDA;
+      if (cur != pl->device && cudaSetDevice(pl->device) != cudaSuccess) return AUGTREE_ERR_CUDA;
+      void *ptr = nullptr;
+      const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+      if (cur != pl->device) cudaSetDevice(cur);
+      if (e != cudaSuccess || !ptr) return AUGTREE_ERR_CUDA;
+      g_static_ptr[pl->device] = ptr;
+    }
+    scratch = g_static_ptr[pl->device];
+  }
+  return augtree_replay_fwd(pl, q_r, k_r, v_r, k_p, v_p, o_r, lse_r, scratch, AUGTREE_STATIC_SCRATCH_BYTES, stream);
 }
 
 int augtree_replay_bwd(const augtree_plan_t *pl, const void *q_r, const void *k_r, const void *v_r, const void *k_p,
