@@ -89,8 +89,8 @@ enum {
   AUGTREE_TBL_REPLAY_FWD_ITEMS = 6,  AUGTREE_TBL_REPLAY_FWD_LANE_PTR = 7,  AUGTREE_TBL_REPLAY_FWD_ORDER = 8,
   AUGTREE_TBL_REPLAY_BWD_ITEMS = 9,  AUGTREE_TBL_REPLAY_BWD_LANE_PTR = 10, AUGTREE_TBL_REPLAY_BWD_ORDER = 11,
   AUGTREE_TBL_PREFILL_BWD_ITEMS = 12, AUGTREE_TBL_PREFILL_BWD_LANE_PTR = 13, AUGTREE_TBL_PREFILL_BWD_ORDER = 14,
-  AUGTREE_TBL_REPLAY_SEGMENTS = 15,  /* [n_branches][2] {first response token, length}      */
-  AUGTREE_TBL_PREFILL_SEGMENTS = 16, /* [n_groups][2]   {first prompt token, length}        */
+  AUGTREE_TBL_REPLAY_SEGMENTS = 15,  /* [n_branches][3] {first response token, length, first query-tile index} */
+  AUGTREE_TBL_PREFILL_SEGMENTS = 16, /* [n_groups][3]   {first prompt token, length, first query-tile index}   */
   AUGTREE_TBL_GROUP_SPLITS = 17,     /* [n_groups] prompt-KV shards actually used           */
   AUGTREE_TBL_COUNT = 18
 };

@@ -80,8 +80,11 @@ def build_tables(prompt_len, branch_len, h_q, h_kv, kv_splits=1):
         "cu_p": np.asarray(cu_p, np.int32), "cu_b": np.asarray(cu_b, np.int32), "cu_r": np.asarray(cu_r, np.int32),
         "prefill_fwd": arr(pf, 12), "replay_fwd": arr(rf, 12), "replay_bwd": arr(rb, 8), "prefill_bwd": arr(pb, 8),
         "group_splits": np.asarray(gsplits, np.int32),
-        "seg_replay": np.asarray([[cu_r[i], flat[i]] for i in range(len(flat))], np.int32).reshape(-1, 2),
-        "seg_prefill": np.asarray([[cu_p[g], prompt_len[g]] for g in range(len(prompt_len))], np.int32).reshape(-1, 2),
+        # segments: first token, length, index of the segment's first 128-row query tile
+        "seg_replay": np.asarray([[cu_r[i], flat[i], sum(_cdiv(x, TQ) for x in flat[:i])] for i in range(len(flat))],
+                                 np.int32).reshape(-1, 3),
+        "seg_prefill": np.asarray([[cu_p[g], prompt_len[g], sum(_cdiv(x, TQ) for x in prompt_len[:g])]
+                                   for g in range(len(prompt_len))], np.int32).reshape(-1, 3),
     }
 
 

@@ -59,6 +59,21 @@ int make_map(CUtensorMap *m, const void *ptr, long long tokens, int heads, int d
   return r == CUDA_SUCCESS ? AUGTREE_OK : AUGTREE_ERR_CUDA;
 }
 
+// Tensor map over the fp32 dQ accumulator [tokens, heads, d]: boxes of 32 tokens
+// by 32 floats (128 bytes) of one head, 128-byte swizzle, used for reduce-adds.
+int make_map_f32(CUtensorMap *m, void *ptr, long long tokens, int heads, int d) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return AUGTREE_ERR_CUDA;
+  if (tokens < 1) tokens = 1;
+  const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)heads, (cuuint64_t)tokens};
+  const cuuint64_t strides[2] = {(cuuint64_t)d * 4, (cuuint64_t)heads * d * 4};
+  const cuuint32_t box[3] = {32, 1, 32};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+}
+
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 size_t al256(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -123,6 +138,8 @@ struct BwdArgs {
   float *dk_acc, *dv_acc;
   int causal_fp32;
   const int32_t *d_segs;
+  const int32_t *d_tiles;  // [n_tiles][2] query tiles of the call's query tensor
+  long long n_tiles;
 };
 
 template <int D>
@@ -134,20 +151,16 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
   float *dq_acc = reinterpret_cast<float *>(w);
   // region sizes must match build_plan_host: sized for max(total_p, total_r)
   const size_t tmax = (size_t)(pl->total_p > pl->total_r ? pl->total_p : pl->total_r);
-  float *delta = reinterpret_cast<float *>(w + al256(tmax * hq * D * 4));
-  float *lse2 = reinterpret_cast<float *>(w + al256(tmax * hq * D * 4) + al256(tmax * hq * 4));
+  float *stats = reinterpret_cast<float *>(w + al256(tmax * hq * D * 4));
   if (cudaMemsetAsync(dq_acc, 0, n_el * 4, st) != cudaSuccess) return AUGTREE_ERR_CUDA;
   {
-    const long long warps = a.q_tok * (long long)hq;
-    const int threads = 256;
-    const long long blocks = (warps * 32 + threads - 1) / threads;
-    bwd_preprocess_kernel<D><<<(unsigned)blocks, threads, 0, st>>>(
-        static_cast<const __nv_bfloat16 *>(a.o), static_cast<const __nv_bfloat16 *>(a.d_o), a.lse, delta, lse2, a.q_tok,
-        pl->h_q);
+    const dim3 grid((unsigned)a.n_tiles, (unsigned)pl->h_q);
+    bwd_preprocess_kernel<D><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(a.o), static_cast<const __nv_bfloat16 *>(a.d_o),
+                                                   a.lse, a.d_tiles, stats, a.q_tok, a.n_tiles, pl->h_q, pl->scale);
     ++g_launches;
   }
   if (s.n_items() > 0) {
-    CUtensorMap mq, mdo, mk0, mv0, mk1, mv1;
+    CUtensorMap mq, mdo, mk0, mv0, mk1, mv1, mdq;
     int r;
     if ((r = make_map(&mq, a.q, a.q_tok, pl->h_q, D))) return r;
     if ((r = make_map(&mdo, a.d_o, a.q_tok, pl->h_q, D))) return r;
@@ -155,10 +168,11 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     if ((r = make_map(&mv0, a.v0, a.kv0_tok, pl->h_kv, D))) return r;
     if ((r = make_map(&mk1, a.k1, a.kv1_tok, pl->h_kv, D))) return r;
     if ((r = make_map(&mv1, a.v1, a.kv1_tok, pl->h_kv, D))) return r;
+    if ((r = make_map_f32(&mdq, dq_acc, a.q_tok, pl->h_q, D))) return r;
     BwdParams p;
-    p.items = s.d_items; p.lane_ptr = s.d_lane_ptr; p.segs = a.d_segs; p.lse2 = lse2; p.delta = delta; p.dq_acc = dq_acc;
+    p.items = s.d_items; p.lane_ptr = s.d_lane_ptr; p.segs = a.d_segs; p.stats = stats;
     p.dk_out = static_cast<__nv_bfloat16 *>(a.dk_out); p.dv_out = static_cast<__nv_bfloat16 *>(a.dv_out);
-    p.dk_acc = a.dk_acc; p.dv_acc = a.dv_acc; p.n_tok = a.q_tok; p.h_q = pl->h_q; p.h_kv = pl->h_kv;
+    p.dk_acc = a.dk_acc; p.dv_acc = a.dv_acc; p.n_tiles = a.n_tiles; p.h_q = pl->h_q; p.h_kv = pl->h_kv;
     p.causal_fp32 = a.causal_fp32; p.scale = pl->scale; p.scale_log2 = pl->scale * 1.4426950408889634f;
     p.status = pl->d_status;
     static bool attr_set[2] = {false, false};
@@ -169,7 +183,7 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     }
     const int kind = (int)(&s - pl->sched);
     timing_mark(pl, kind, false, st);
-    bwd_kernel<D><<<pl->n_lanes, kBwdThreads, BwdSmem<D>::kBytes, st>>>(mq, mdo, mk0, mv0, mk1, mv1, p);
+    bwd_kernel<D><<<pl->n_lanes, kBwdThreads, BwdSmem<D>::kBytes, st>>>(mq, mdo, mk0, mv0, mk1, mv1, mdq, p);
     timing_mark(pl, kind, true, st);
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return AUGTREE_ERR_CUDA;
@@ -237,6 +251,8 @@ int augtree_plan_create(const augtree_desc_t *desc, int device, augtree_plan_t *
     if (!r) r = upload(pl->branch_group, &pl->d_branch_group);
     if (!r) r = upload(pl->group_splits, &pl->d_group_splits);
     if (!r) r = upload(pl->cu_r, &pl->d_cu_r);
+    if (!r) r = upload(pl->tiles_replay, &pl->d_tiles_replay);
+    if (!r) r = upload(pl->tiles_prefill, &pl->d_tiles_prefill);
     if (!r) {
       if (cudaMalloc(&pl->d_status, 2 * sizeof(int)) != cudaSuccess || cudaMemset(pl->d_status, 0, 2 * sizeof(int)) != cudaSuccess)
         r = AUGTREE_ERR_CUDA;
@@ -256,7 +272,7 @@ int augtree_plan_destroy(augtree_plan_t *pl) {
     cudaSetDevice(pl->device);
     for (int k = 0; k < SCHED_COUNT; ++k) { cudaFree(pl->sched[k].d_items); cudaFree(pl->sched[k].d_lane_ptr); }
     cudaFree(pl->d_seg_replay); cudaFree(pl->d_seg_prefill); cudaFree(pl->d_branch_group); cudaFree(pl->d_group_splits);
-    cudaFree(pl->d_cu_r); cudaFree(pl->d_status);
+    cudaFree(pl->d_cu_r); cudaFree(pl->d_status); cudaFree(pl->d_tiles_replay); cudaFree(pl->d_tiles_prefill);
     if (pl->timing) {
       for (int k = 0; k < SCHED_COUNT; ++k)
         for (void *e : pl->timing->ev[k]) cudaEventDestroy(static_cast<cudaEvent_t>(e));
@@ -401,7 +417,7 @@ int augtree_replay_bwd(const augtree_plan_t *pl, const void *q_r, const void *k_
   a.q = q_r; a.d_o = do_r; a.o = o_r; a.lse = lse_r; a.q_tok = pl->total_r;
   a.k0 = k_r; a.v0 = v_r; a.kv0_tok = pl->total_r; a.k1 = k_p; a.v1 = v_p; a.kv1_tok = pl->total_p;
   a.dq = dq_r; a.dk_out = dk_r; a.dv_out = dv_r; a.dk_acc = dkp_acc; a.dv_acc = dvp_acc; a.causal_fp32 = 0;
-  a.d_segs = pl->d_seg_replay;
+  a.d_segs = pl->d_seg_replay; a.d_tiles = pl->d_tiles_replay; a.n_tiles = (long long)pl->tiles_replay.size() / 2;
   const Sched &s = pl->sched[SCHED_REPLAY_BWD];
   return pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, st) : launch_bwd<64>(pl, s, a, ws, st);
 }
@@ -421,7 +437,7 @@ int augtree_prefill_bwd(const augtree_plan_t *pl, const void *q_p, const void *k
   a.q = q_p; a.d_o = do_p; a.o = o_p; a.lse = lse_p; a.q_tok = pl->total_p;
   a.k0 = k_p; a.v0 = v_p; a.kv0_tok = pl->total_p; a.k1 = k_p; a.v1 = v_p; a.kv1_tok = pl->total_p;
   a.dq = dq_p; a.dk_out = nullptr; a.dv_out = nullptr; a.dk_acc = dkp_acc; a.dv_acc = dvp_acc; a.causal_fp32 = 1;
-  a.d_segs = pl->d_seg_prefill;
+  a.d_segs = pl->d_seg_prefill; a.d_tiles = pl->d_tiles_prefill; a.n_tiles = (long long)pl->tiles_prefill.size() / 2;
   const Sched &s = pl->sched[SCHED_PREFILL_BWD];
   r = pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, st) : launch_bwd<64>(pl, s, a, ws, st);
   if (r) return r;

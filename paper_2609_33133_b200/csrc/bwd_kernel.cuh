@@ -6,15 +6,22 @@
 // one TMEM accumulator in a fixed order; for a tile inside a sequence, the
 // causal query tiles of that sequence.
 //
-// Per (KV tile, Q tile, head) pair, with S^T = K Q^T so that a thread owns a key:
-//   P^T = exp2(S^T * scale*log2e - lse2[q]),  dP^T = V dO^T,
-//   dS^T = scale * P^T * (dP^T - delta[q]),
-//   dV += P^T dO,  dK += dS^T Q,  dQ[q,:] += dS K   (dQ leaves through fp32 atomics).
+// Per (KV tile, Q tile, head) pair T, with S^T = K Q^T so that a TMEM lane is a key:
+//   P^T  = exp2(S^T * scale*log2e - lse2[q])          (element-wise warps)
+//   dP^T = V dO^T
+//   dS^T = P^T * (scale*dP^T - scale*delta[q])        (element-wise warps)
+//   dV  += P^T dO      (A = P^T from TMEM)
+//   dK  += dS^T Q      (A = dS^T from shared memory, K-major)
+//   dQ   = dS K        (A = the same dS^T tile read MN-major) -> fp32 TMA reduce-add
 //
-// Warp roles (192 threads): warps 0-3 element-wise work and epilogues, warp 4
-// lane 0 TMA, warp 5 lane 0 MMA.  TMEM columns: T0 [0,128) holds S^T, then P^T
-// (bf16, columns 0-63) and the low half of dQ (columns 64-127); T1 [128,256)
-// holds dP^T, then dS^T and the high half of dQ; dV at 256, dK at 256 + D.
+// Warp roles (320 threads): warps 0-7 element-wise (warp w: TMEM lanes
+// 32*(w%4).., query columns 64*(w/4)..), warp 8 lane 0 TMA loads, warp 9 lane 0
+// MMA issue.  TMEM columns: R0 [0,128) S^T, overwritten in place by P^T (bf16);
+// R1 [128,256) dP^T, later dQ; dV at 256; dK at 256 + D.
+//
+// MMA issue order in steady state: dP(T), S(T+1), dK(T), dQ(T), dV(T+1), so the
+// tensor pipe has independent work while the warps turn S into P, dP into dS
+// and drain dQ.
 #pragma once
 #include <cuda.h>
 
@@ -25,74 +32,98 @@ namespace augtree {
 struct BwdParams {
   const int32_t *items;     // lane order, 8 ints each
   const int32_t *lane_ptr;  // [gridDim.x + 1]
-  const int32_t *segs;      // [n_seg][2] {first query token, length}
-  const float *lse2;        // [h_q, n_tok]  lse * log2(e)
-  const float *delta;       // [h_q, n_tok]  rowsum(dO * O)
-  float *dq_acc;            // [n_tok, h_q, D] fp32, zeroed by the caller
+  const int32_t *segs;      // [n_seg][3] {first query token, length, first tile index}
+  const float *stats;       // [h_q][n_tiles][2][128]: lse*log2e (inf past the end), scale*rowsum(dO*O)
   __nv_bfloat16 *dk_out, *dv_out;  // mode-0 items when causal_fp32 == 0: [kv tokens, h_kv, D] bf16
   float *dk_acc, *dv_acc;   // fp32 [prompt tokens, h_kv, D]: mode-1 items, and mode-0 items when causal_fp32 != 0
-  long long n_tok;          // tokens of the query tensor
+  long long n_tiles;        // query tiles in the stats table
   int h_q, h_kv;
   int causal_fp32;
   float scale, scale_log2;
   int *status;
 };
 
-constexpr int kBwdThreads = 192;
+constexpr int kBwdThreads = 320;
 constexpr int kBwdStages = 2;
 
 template <int D>
 struct BwdSmem {
   static constexpr int kTileBytes = 128 * D * 2;
   static constexpr int kDsBytes = 128 * 128 * 2;
-  static constexpr int kOffK = 0, kOffV = kTileBytes, kOffQ = 2 * kTileBytes;  // Q[s], dO[s] interleaved per stage
-  static constexpr int kOffDs = kOffQ + 2 * kBwdStages * kTileBytes;
-  static constexpr int kOffRow = kOffDs + kDsBytes;  // lse2[128], delta[128] of the current query tile
-  static constexpr int kOffBar = kOffRow + 2 * 128 * 4;
-  static constexpr int kBytes = kOffBar + 160 + 1024;
+  static constexpr int kOffK = 0, kOffV = kTileBytes;
+  static constexpr int kOffQ = 2 * kTileBytes;                        // [kBwdStages]
+  static constexpr int kOffDo = kOffQ + kBwdStages * kTileBytes;      // [kBwdStages]
+  static constexpr int kOffDs = kOffDo + kBwdStages * kTileBytes;     // dS^T tile, reused as dQ staging
+  static constexpr int kOffStats = kOffDs + kDsBytes;                 // [kBwdStages][2][128] floats
+  static constexpr int kOffBar = kOffStats + kBwdStages * 1024;
+  static constexpr int kBytes = kOffBar + 256;
 };
+
+// bulk copy global -> shared (1-D), completion on an mbarrier
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// fp32 reduce-add of a shared-memory box into a global tensor
+__device__ __forceinline__ void tma_reduce_add_3d(const void *tmap, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(tmap), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
            const __grid_constant__ CUtensorMap tm_k0, const __grid_constant__ CUtensorMap tm_v0,
-           const __grid_constant__ CUtensorMap tm_k1, const __grid_constant__ CUtensorMap tm_v1, const BwdParams p) {
+           const __grid_constant__ CUtensorMap tm_k1, const __grid_constant__ CUtensorMap tm_v1,
+           const __grid_constant__ CUtensorMap tm_dq, const BwdParams p) {
   using SM = BwdSmem<D>;
   constexpr int TILE = SM::kTileBytes;
   constexpr int NBOX = D / 64;
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t sK = base + SM::kOffK, sV = base + SM::kOffV, sQ0 = base + SM::kOffQ, sDs = base + SM::kOffDs;
-  float *rb = reinterpret_cast<float *>(gen + SM::kOffRow);  // [2][128]
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t base = smem_u32(smem_raw);
+  if (base & 1023u) {  // the 128-byte swizzle needs 1024-byte aligned tiles
+    if (threadIdx.x == 0 && atomicCAS(p.status, 0, -6) == 0) p.status[1] = 1;
+    return;
+  }
+  const uint32_t sK = base + SM::kOffK, sV = base + SM::kOffV, sQ0 = base + SM::kOffQ, sDo0 = base + SM::kOffDo;
+  const uint32_t sDs = base + SM::kOffDs, sStats0 = base + SM::kOffStats;
   const uint32_t bars = base + SM::kOffBar;
   const uint32_t bar_kv_full = bars, bar_kv_empty = bars + 8;
-  const uint32_t bar_qdo_full = bars + 16, bar_qdo_empty = bars + 32;  // [2] each
-  const uint32_t bar_s_full = bars + 48, bar_pds_full = bars + 56, bar_mma2 = bars + 64, bar_dq_free = bars + 72;
-  const uint32_t bar_acc_full = bars + 80, bar_acc_empty = bars + 88, bar_rows = bars + 96;
-  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen + SM::kOffBar + 104);
-  volatile int *abort_flag = reinterpret_cast<volatile int *>(gen + SM::kOffBar + 112);
+  const uint32_t bar_q_full = bars + 16, bar_q_empty = bars + 32;    // [2] each
+  const uint32_t bar_do_full = bars + 48, bar_do_empty = bars + 64;  // [2] each
+  const uint32_t bar_s_full = bars + 80, bar_p_ready = bars + 88, bar_dp_full = bars + 96, bar_ds_ready = bars + 104;
+  const uint32_t bar_dq_full = bars + 112, bar_drained = bars + 120, bar_stage_free = bars + 128;
+  const uint32_t bar_acc_full = bars + 136, bar_acc_empty = bars + 144;
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_raw + SM::kOffBar + 160);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + SM::kOffBar + 168);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     mbar_init(bar_kv_full, 1); mbar_init(bar_kv_empty, 1);
-    for (int s = 0; s < kBwdStages; ++s) { mbar_init(bar_qdo_full + 8 * s, 1); mbar_init(bar_qdo_empty + 8 * s, 1); }
-    mbar_init(bar_s_full, 1); mbar_init(bar_pds_full, 128); mbar_init(bar_mma2, 1); mbar_init(bar_dq_free, 128);
-    mbar_init(bar_acc_full, 1); mbar_init(bar_acc_empty, 128); mbar_init(bar_rows, 128);
+    for (int s = 0; s < kBwdStages; ++s) {
+      mbar_init(bar_q_full + 8 * s, 1); mbar_init(bar_q_empty + 8 * s, 1);
+      mbar_init(bar_do_full + 8 * s, 1); mbar_init(bar_do_empty + 8 * s, 1);
+    }
+    mbar_init(bar_s_full, 1); mbar_init(bar_p_ready, 256); mbar_init(bar_dp_full, 1); mbar_init(bar_ds_ready, 256);
+    mbar_init(bar_dq_full, 1); mbar_init(bar_drained, 256); mbar_init(bar_stage_free, 8);
+    mbar_init(bar_acc_full, 1); mbar_init(bar_acc_empty, 256);
     *abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == 5) { tmem_alloc(smem_u32((const void *)tmem_slot), 512); tmem_relinquish(); }
+  if (warp == 9) { tmem_alloc(smem_u32((const void *)tmem_slot), 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tT0 = tmem, tT1 = tmem + 128, tDV = tmem + 256, tDK = tmem + 256 + D;
+  const uint32_t tR0 = tmem, tR1 = tmem + 128, tDV = tmem + 256, tDK = tmem + 256 + D;
   const AbortCtx ab{abort_flag, p.status};
   const int rep = p.h_q / p.h_kv;
   const int it_begin = p.lane_ptr[blockIdx.x], it_end = p.lane_ptr[blockIdx.x + 1];
 
-  if (warp == 4) {
+  if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_do); tma_prefetch_desc(&tm_k0);
@@ -112,85 +143,116 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           tma_load_3d(sV + b * 16384, mode ? &tm_v1 : &tm_v0, bar_kv_full, b * 64, kvh, kv_tok0);
         }
         for (int sg = seg0; sg < seg0 + nseg && ok; ++sg) {
-          const int s_tok0 = p.segs[2 * sg], s_len = p.segs[2 * sg + 1];
+          const int s_tok0 = p.segs[3 * sg], s_len = p.segs[3 * sg + 1], s_tile0 = p.segs[3 * sg + 2];
           const int nqt = (s_len + 127) >> 7;
           for (int qt = mode ? 0 : (kv_pos0 >> 7); qt < nqt && ok; ++qt)
             for (int j = 0; j < rep; ++j, ++T) {
               const uint32_t st = T % kBwdStages, par = ((T / kBwdStages) & 1) ^ 1;
-              ok = mbar_wait(bar_qdo_empty + 8 * st, par, ab, WAIT_BWD_QDO_EMPTY);
+              const int head = kvh * rep + j, row = s_tok0 + qt * 128;
+              ok = mbar_wait(bar_q_empty + 8 * st, par, ab, WAIT_BWD_QDO_EMPTY);
               if (!ok) break;
-              mbar_expect_tx(bar_qdo_full + 8 * st, 2 * TILE);
-              const uint32_t dq = sQ0 + st * 2 * TILE, ddo = dq + TILE;
-              for (int b = 0; b < NBOX; ++b) {
-                tma_load_3d(dq + b * 16384, &tm_q, bar_qdo_full + 8 * st, b * 64, kvh * rep + j, s_tok0 + qt * 128);
-                tma_load_3d(ddo + b * 16384, &tm_do, bar_qdo_full + 8 * st, b * 64, kvh * rep + j, s_tok0 + qt * 128);
-              }
+              mbar_expect_tx(bar_q_full + 8 * st, TILE + 1024);
+              for (int b = 0; b < NBOX; ++b) tma_load_3d(sQ0 + st * TILE + b * 16384, &tm_q, bar_q_full + 8 * st, b * 64, head, row);
+              bulk_load_1d(sStats0 + st * 1024, p.stats + ((long long)head * p.n_tiles + s_tile0 + qt) * 256, 1024,
+                           bar_q_full + 8 * st);
+              ok = mbar_wait(bar_do_empty + 8 * st, par, ab, WAIT_BWD_QDO_EMPTY);
+              if (!ok) break;
+              mbar_expect_tx(bar_do_full + 8 * st, TILE);
+              for (int b = 0; b < NBOX; ++b) tma_load_3d(sDo0 + st * TILE + b * 16384, &tm_do, bar_do_full + 8 * st, b * 64, head, row);
             }
         }
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       constexpr uint32_t IDESC_ST = make_idesc(128, 128, 0, 0);  // S^T, dP^T: both operands K-major
-      constexpr uint32_t IDESC_ACC = make_idesc(128, D, 0, 1);   // dV, dK: A from TMEM, B = dO / Q MN-major
-      constexpr uint32_t IDESC_DQ = make_idesc(128, 64, 1, 1);   // dQ halves: A = dS MN-major, B = K MN-major
+      constexpr uint32_t IDESC_DV = make_idesc(128, D, 0, 1);    // dV: A = P^T (TMEM), B = dO MN-major
+      constexpr uint32_t IDESC_DK = make_idesc(128, D, 0, 1);    // dK: A = dS^T K-major (shared), B = Q MN-major
+      constexpr uint32_t IDESC_DQ = make_idesc(128, D, 1, 1);    // dQ: A = dS^T read MN-major, B = K MN-major
       uint32_t ic = 0, T = 0;
       bool ok = true;
+      auto issue_s = [&](uint32_t Tn) -> bool {  // S^T(Tn) = K Q^T -> R0
+        const uint32_t st = Tn % kBwdStages;
+        if (!mbar_wait(bar_q_full + 8 * st, (Tn / kBwdStages) & 1, ab, WAIT_BWD_QDO_FULL)) return false;
+        tc_fence_after();
+        const uint32_t sQ = sQ0 + st * TILE;
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
+          mma_ss(tR0, make_sdesc(sK + off, 16, 1024), make_sdesc(sQ + off, 16, 1024), IDESC_ST, k > 0);
+        }
+        tc_commit(bar_s_full);
+        return true;
+      };
+      auto issue_dv = [&](uint32_t Tn, uint32_t acc0) -> bool {  // dV += P^T(Tn) dO(Tn)
+        const uint32_t st = Tn % kBwdStages;
+        if (!mbar_wait(bar_p_ready, Tn & 1, ab, WAIT_BWD_PDS_FULL)) return false;
+        if (!mbar_wait(bar_do_full + 8 * st, (Tn / kBwdStages) & 1, ab, WAIT_BWD_QDO_FULL)) return false;
+        tc_fence_after();
+        const uint32_t sdO = sDo0 + st * TILE;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)  // query columns 16k..16k+15: P^T sits at R0 columns 8k (k<4) or 64+8(k-4)
+          mma_ts(tDV, tR0 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), make_sdesc(sdO + k * 2048, 16384, 1024), IDESC_DV,
+                 acc0 | (uint32_t)(k > 0));
+        return true;
+      };
       for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
         const int32_t *I = p.items + (size_t)it * 8;
         const int kv_pos0 = I[1], mode = I[4], seg0 = I[5], nseg = I[6];
+        int n_pairs = 0;
+        for (int sg = seg0; sg < seg0 + nseg; ++sg) {
+          const int nqt = (p.segs[3 * sg + 1] + 127) >> 7;
+          n_pairs += (nqt - (mode ? 0 : (kv_pos0 >> 7))) * rep;
+        }
         ok = mbar_wait(bar_kv_full, ic & 1, ab, WAIT_BWD_KV_FULL);
         if (!ok) break;
-        bool first = true;
-        for (int sg = seg0; sg < seg0 + nseg && ok; ++sg) {
-          const int nqt = (p.segs[2 * sg + 1] + 127) >> 7;
-          for (int qt = mode ? 0 : (kv_pos0 >> 7); qt < nqt && ok; ++qt)
-            for (int j = 0; j < rep; ++j, ++T) {
-              const uint32_t st = T % kBwdStages;
-              const uint32_t sQ = sQ0 + st * 2 * TILE, sdO = sQ + TILE;
-              ok = mbar_wait(bar_qdo_full + 8 * st, (T / kBwdStages) & 1, ab, WAIT_BWD_QDO_FULL);
-              if (!ok) break;
-              if (T > 0) {
-                ok = mbar_wait(bar_dq_free, (T - 1) & 1, ab, WAIT_BWD_DQ_FREE);
-                if (!ok) break;
-              }
-              tc_fence_after();
+        // prologue: S(T), dV(T) of the item's first pair
+        ok = issue_s(T);
+        if (!ok) break;
+        if (ic > 0) {
+          ok = mbar_wait(bar_acc_empty, (ic - 1) & 1, ab, WAIT_BWD_ACC_EMPTY);
+          if (!ok) break;
+        }
+        ok = issue_dv(T, 0u);
+        for (int i = 0; i < n_pairs && ok; ++i, ++T) {
+          const uint32_t st = T % kBwdStages;
+          const uint32_t sQ = sQ0 + st * TILE, sdO = sDo0 + st * TILE;
+          // dP^T(T) = V dO^T -> R1 (needs dQ(T-1) drained out of R1)
+          if (T > 0) {
+            ok = mbar_wait(bar_drained, (T - 1) & 1, ab, WAIT_BWD_DQ_FREE);
+            if (!ok) break;
+          }
+          tc_fence_after();
 #pragma unroll
-              for (int k = 0; k < D / 16; ++k) {
-                const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-                mma_ss(tT0, make_sdesc(sK + off, 16, 1024), make_sdesc(sQ + off, 16, 1024), IDESC_ST, k > 0);
-              }
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
+            mma_ss(tR1, make_sdesc(sV + off, 16, 1024), make_sdesc(sdO + off, 16, 1024), IDESC_ST, k > 0);
+          }
+          tc_commit(bar_dp_full);
+          tc_commit(bar_do_empty + 8 * st);  // dO(T) was last read by dV(T) (issued earlier) and dP(T)
+          // S^T(T+1)
+          if (i + 1 < n_pairs) {
+            ok = issue_s(T + 1);
+            if (!ok) break;
+          }
+          // dK += dS^T(T) Q(T);  dQ(T) = dS(T) K -> R1
+          ok = mbar_wait(bar_ds_ready, T & 1, ab, WAIT_BWD_PDS_FULL);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t acc0 = i > 0 ? 1u : 0u;
 #pragma unroll
-              for (int k = 0; k < D / 16; ++k) {
-                const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-                mma_ss(tT1, make_sdesc(sV + off, 16, 1024), make_sdesc(sdO + off, 16, 1024), IDESC_ST, k > 0);
-              }
-              tc_commit(bar_s_full);
-              ok = mbar_wait(bar_pds_full, T & 1, ab, WAIT_BWD_PDS_FULL);
-              if (!ok) break;
-              if (first && ic > 0) {
-                ok = mbar_wait(bar_acc_empty, (ic - 1) & 1, ab, WAIT_BWD_ACC_EMPTY);
-                if (!ok) break;
-              }
-              tc_fence_after();
-              const uint32_t acc0 = first ? 0u : 1u;
+          for (int k = 0; k < 8; ++k) {  // K dim = 128 queries: dS^T box k/4, 32 bytes per step
+            const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
+            mma_ss(tDK, make_sdesc(sDs + off, 16, 1024), make_sdesc(sQ + k * 2048, 16384, 1024), IDESC_DK, acc0 | (uint32_t)(k > 0));
+          }
+          tc_commit(bar_q_empty + 8 * st);
 #pragma unroll
-              for (int k = 0; k < 8; ++k)
-                mma_ts(tDV, tT0 + k * 8, make_sdesc(sdO + k * 2048, 16384, 1024), IDESC_ACC, acc0 | (k > 0));
-#pragma unroll
-              for (int k = 0; k < 8; ++k)
-                mma_ts(tDK, tT1 + k * 8, make_sdesc(sQ + k * 2048, 16384, 1024), IDESC_ACC, acc0 | (k > 0));
-#pragma unroll
-              for (int h = 0; h < NBOX; ++h)
-#pragma unroll
-                for (int k = 0; k < 8; ++k)
-                  mma_ss((h ? tT1 : tT0) + 64, make_sdesc(sDs + k * 2048, 16384, 1024),
-                         make_sdesc(sK + h * 16384 + k * 2048, 16384, 1024), IDESC_DQ, k > 0);
-              tc_commit(bar_mma2);
-              tc_commit(bar_qdo_empty + 8 * st);
-              first = false;
-            }
+          for (int k = 0; k < 8; ++k)  // K dim = 128 keys: 16 rows of dS^T / K per step
+            mma_ss(tR1, make_sdesc(sDs + k * 2048, 16384, 1024), make_sdesc(sK + k * 2048, 16384, 1024), IDESC_DQ, k > 0);
+          tc_commit(bar_dq_full);
+          // dV += P^T(T+1) dO(T+1)
+          if (i + 1 < n_pairs) ok = issue_dv(T + 1, 1u);
         }
         if (!ok) break;
         tc_commit(bar_acc_full);
@@ -198,116 +260,187 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       }
     }
   } else {
-    // ------------------------------------------------------- compute warps 0-3
-    const int t = threadIdx.x;  // TMEM lane: key row for S^T/dP^T/dV/dK, query row for dQ
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    // ------------------------------------------------------- element-wise warps 0-7
+    const int lg = warp & 3, ch = warp >> 2;
+    const int r = lg * 32 + lane;  // TMEM lane: key row for S^T/dP^T/dV/dK, query row for dQ
+    const uint32_t lane_off = (uint32_t)(lg * 32) << 16;
+    const uint32_t stage_buf = sDs + warp * 4096;  // this warp's 32 x 128-byte dQ staging rows
+    uint8_t *stage_gen = smem_raw + SM::kOffDs + warp * 4096;
     uint32_t ic = 0, T = 0;
     bool ok = true;
+    float pr[64];  // P^T of the current pair: key r, query columns 64*ch .. 64*ch+63
+
+    // P^T(Tn) from S^T(Tn): wait, load, exponentiate, store bf16 over S^T, signal
+    auto make_p = [&](uint32_t Tn, int q_base, int kv_pos0, int mode, bool key_valid) -> bool {
+      const uint32_t st = Tn % kBwdStages;
+      if (!mbar_wait(bar_q_full + 8 * st, (Tn / kBwdStages) & 1, ab, WAIT_BWD_QDO_FULL)) return false;  // row statistics landed
+      if (!mbar_wait(bar_s_full, Tn & 1, ab, WAIT_BWD_S_FULL)) return false;
+      tc_fence_after();
+      const float *lse2 = reinterpret_cast<const float *>(smem_raw + SM::kOffStats + st * 1024) + ch * 64;
+      // query column (inside the tile) from which this key is visible
+      const int lo = mode ? 0 : (kv_pos0 + r - q_base);
+      const bool all_visible = key_valid && lo <= ch * 64;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t sv[32];
+        tmem_ld32(tR0 + lane_off + ch * 64 + c * 32, sv);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + c * 32 + i);
+          pr[c * 32 + i + 0] = ex2(__uint_as_float(sv[i + 0]) * p.scale_log2 - l4.x);
+          pr[c * 32 + i + 1] = ex2(__uint_as_float(sv[i + 1]) * p.scale_log2 - l4.y);
+          pr[c * 32 + i + 2] = ex2(__uint_as_float(sv[i + 2]) * p.scale_log2 - l4.z);
+          pr[c * 32 + i + 3] = ex2(__uint_as_float(sv[i + 3]) * p.scale_log2 - l4.w);
+        }
+      }
+      if (!all_visible) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i)
+          if (!key_valid || ch * 64 + i < lo) pr[i] = 0.f;
+      }
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(pr[c * 32 + 2 * i], pr[c * 32 + 2 * i + 1]);
+        tmem_st16(tR0 + lane_off + ch * 64 + c * 16, pk);
+      }
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_p_ready);
+      return true;
+    };
+
     for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
       const int32_t *I = p.items + (size_t)it * 8;
       const int kv_tok0 = I[0], kv_pos0 = I[1], kv_rows = I[2], kvh = I[3], mode = I[4], seg0 = I[5], nseg = I[6];
-      const bool key_valid = t < kv_rows;
+      const bool key_valid = r < kv_rows;
+      bool first = true;
       for (int sg = seg0; sg < seg0 + nseg && ok; ++sg) {
-        const int s_tok0 = p.segs[2 * sg], s_len = p.segs[2 * sg + 1];
+        const int s_tok0 = p.segs[3 * sg], s_len = p.segs[3 * sg + 1];
         const int nqt = (s_len + 127) >> 7;
-        for (int qt = mode ? 0 : (kv_pos0 >> 7); qt < nqt && ok; ++qt)
+        const int qt0 = mode ? 0 : (kv_pos0 >> 7);
+        for (int qt = qt0; qt < nqt && ok; ++qt)
           for (int j = 0; j < rep; ++j, ++T) {
-            const int head = kvh * rep + j;
-            const int q_rows = min(128, s_len - qt * 128);
-            const long long tok = (long long)s_tok0 + qt * 128 + t;
-            {
-              const bool qv = t < q_rows;
-              rb[t] = qv ? p.lse2[(long long)head * p.n_tok + tok] : INFINITY;
-              rb[128 + t] = qv ? p.delta[(long long)head * p.n_tok + tok] : 0.f;
+            const uint32_t st = T % kBwdStages;
+            if (first) {  // the item's first pair has no predecessor to pipeline behind
+              ok = make_p(T, qt * 128, kv_pos0, mode, key_valid);
+              if (!ok) break;
+              first = false;
             }
-            mbar_arrive(bar_rows);
-            ok = mbar_wait(bar_rows, T & 1, ab, WAIT_BWD_ROWS);
+            // ---- dS^T(T) = P^T * (scale*dP^T - scale*delta): to shared memory (K-major rows of 64 queries)
+            ok = mbar_wait(bar_dp_full, T & 1, ab, WAIT_BWD_S_FULL);
             if (!ok) break;
-            ok = mbar_wait(bar_s_full, T & 1, ab, WAIT_BWD_S_FULL);
-            if (!ok) break;
+            if (T > 0) {  // the dQ staging of pair T-1 shares the dS^T buffer
+              ok = mbar_wait(bar_stage_free, (T - 1) & 1, ab, WAIT_BWD_ROWS);
+              if (!ok) break;
+            }
             tc_fence_after();
-            // first query column this key may NOT be hidden from: col >= lo is visible
-            const int lo = mode ? 0 : (kv_pos0 + t - qt * 128);
+            {
+              const float *dl = reinterpret_cast<const float *>(smem_raw + SM::kOffStats + st * 1024) + 128 + ch * 64;
+              uint8_t *row = smem_raw + SM::kOffDs + ch * 16384 + r * 128;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              uint32_t sv[32], dpv[32];
-              tmem_ld32(tT0 + lane_off + c * 32, sv);
-              tmem_ld32(tT1 + lane_off + c * 32, dpv);
-              tc_wait_ld();
-              uint32_t pp[16], dd[16];
+              for (int c = 0; c < 2; ++c) {
+                uint32_t dpv[32];
+                tmem_ld32(tR1 + lane_off + ch * 64 + c * 32, dpv);
+                tc_wait_ld();
+                uint32_t dd[16];
 #pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                float pv[2], dv[2];
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                  const int col = c * 32 + 2 * i + e;
-                  const float l2 = rb[col], dl = rb[128 + col];
-                  float pr = ex2(__uint_as_float(sv[2 * i + e]) * p.scale_log2 - l2);
-                  if (!key_valid || col < lo) pr = 0.f;
-                  pv[e] = pr;
-                  dv[e] = pr * (__uint_as_float(dpv[2 * i + e]) - dl) * p.scale;
+                for (int i = 0; i < 32; i += 4) {
+                  const float4 d4 = *reinterpret_cast<const float4 *>(dl + c * 32 + i);
+                  const float a0 = pr[c * 32 + i + 0] * fmaf(__uint_as_float(dpv[i + 0]), p.scale, -d4.x);
+                  const float a1 = pr[c * 32 + i + 1] * fmaf(__uint_as_float(dpv[i + 1]), p.scale, -d4.y);
+                  const float a2 = pr[c * 32 + i + 2] * fmaf(__uint_as_float(dpv[i + 2]), p.scale, -d4.z);
+                  const float a3 = pr[c * 32 + i + 3] * fmaf(__uint_as_float(dpv[i + 3]), p.scale, -d4.w);
+                  dd[i / 2] = pack_bf16(a0, a1);
+                  dd[i / 2 + 1] = pack_bf16(a2, a3);
                 }
-                pp[i] = pack_bf16(pv[0], pv[1]);
-                dd[i] = pack_bf16(dv[0], dv[1]);
-              }
-              tmem_st16(tT0 + lane_off + c * 16, pp);
-              tmem_st16(tT1 + lane_off + c * 16, dd);
-              // dS^T row t, query columns [32c, 32c+32) -> shared, MN-major (query contiguous), 128B swizzle
-              uint8_t *row = gen + SM::kOffDs + (c >> 1) * 16384 + t * 128;
 #pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                const int chunk = (c & 1) * 4 + v;
-                *reinterpret_cast<uint4 *>(row + ((chunk ^ (t & 7)) << 4)) =
-                    make_uint4(dd[4 * v], dd[4 * v + 1], dd[4 * v + 2], dd[4 * v + 3]);
+                for (int v = 0; v < 4; ++v) {
+                  const int chunk = c * 4 + v;
+                  *reinterpret_cast<uint4 *>(row + ((chunk ^ (r & 7)) << 4)) = make_uint4(dd[4 * v], dd[4 * v + 1], dd[4 * v + 2], dd[4 * v + 3]);
+                }
               }
             }
-            tc_wait_st();
             fence_proxy_async_smem();
             tc_fence_before();
-            mbar_arrive(bar_pds_full);
-            // ---- drain dQ of this pair: thread t owns query row t
-            ok = mbar_wait(bar_mma2, T & 1, ab, WAIT_BWD_MMA2);
+            mbar_arrive(bar_ds_ready);
+            // ---- P^T(T+1), if the item has another pair (same iteration order as the other roles)
+            {
+              int nqt2 = qt, j2 = j + 1, sg2 = sg;
+              bool more = true;
+              if (j2 == rep) { j2 = 0; ++nqt2; }
+              int q_base2 = nqt2 * 128;
+              if (nqt2 >= nqt) {
+                ++sg2;
+                if (sg2 < seg0 + nseg) q_base2 = qt0 * 128; else more = false;
+              }
+              if (more) {
+                ok = make_p(T + 1, q_base2, kv_pos0, mode, key_valid);
+                if (!ok) break;
+              }
+            }
+            // ---- drain dQ(T): thread = query row r, columns 64*ch.. of d; fp32 reduce-add by TMA
+            ok = mbar_wait(bar_dq_full, T & 1, ab, WAIT_BWD_MMA2);
             if (!ok) break;
             tc_fence_after();
             {
-              const bool qv = t < q_rows;
-              float *dst = p.dq_acc + (tok * p.h_q + head) * D;
+              const int head = kvh * rep + j;
+              const int tok_row = s_tok0 + qt * 128 + lg * 32;
+              constexpr int ROUNDS = D / 64;  // each round: 32 columns per warp
 #pragma unroll
-              for (int h = 0; h < NBOX; ++h)
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                  uint32_t v[32];
-                  tmem_ld32((h ? tT1 : tT0) + lane_off + 64 + c * 32, v);
-                  tc_wait_ld();
-                  if (qv) {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                      red_add_v4(dst + h * 64 + c * 32 + 4 * i, __uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                 __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
-                  }
+              for (int rd = 0; rd < ROUNDS; ++rd) {
+                const int col0 = (ROUNDS == 2) ? ch * 64 + rd * 32 : ch * 32;
+                uint32_t v[32];
+                tmem_ld32(tR1 + lane_off + col0, v);
+                tc_wait_ld();
+                if (rd == ROUNDS - 1) {  // R1 fully read by this thread: dP(T+1) may overwrite it
+                  tc_fence_before();
+                  mbar_arrive(bar_drained);
                 }
+                if (rd > 0) {  // staging rows still being read by the previous round's reduce
+                  if (lane == 0) bulk_wait_read0();
+                  __syncwarp();
+                }
+                uint8_t *srow = stage_gen + lane * 128;
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                  *reinterpret_cast<uint4 *>(srow + ((q ^ (lane & 7)) << 4)) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                  tma_reduce_add_3d(&tm_dq, stage_buf, col0, head, tok_row);
+                  bulk_commit();
+                }
+              }
+              if (lane == 0) {
+                bulk_wait_read0();
+                mbar_arrive(bar_stage_free);
+              }
+              __syncwarp();
             }
-            tc_fence_before();
-            mbar_arrive(bar_dq_free);
           }
       }
       if (!ok) break;
-      // ---- item epilogue: dV, dK of key row t
+      // ---- item epilogue: dV, dK of key row r, columns 64*ch.. (D = 128) or 32*ch.. (D = 64)
       ok = mbar_wait(bar_acc_full, ic & 1, ab, WAIT_BWD_ACC_FULL);
       if (!ok) break;
       tc_fence_after();
-      const long long krow = ((long long)kv_tok0 + t) * p.h_kv + kvh;
+      const long long krow = ((long long)kv_tok0 + r) * p.h_kv + kvh;
       const bool to_fp32 = mode || p.causal_fp32;
+      constexpr int HALF = D / 2;
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
+        for (int c = 0; c < HALF / 32; ++c) {
+          const int col0 = ch * HALF + c * 32;
           uint32_t v[32];
-          tmem_ld32((which ? tDK : tDV) + lane_off + c * 32, v);
+          tmem_ld32((which ? tDK : tDV) + lane_off + col0, v);
           tc_wait_ld();
           if (key_valid) {
             if (to_fp32) {
-              float4 *dst = reinterpret_cast<float4 *>((which ? p.dk_acc : p.dv_acc) + krow * D + c * 32);
+              float4 *dst = reinterpret_cast<float4 *>((which ? p.dk_acc : p.dv_acc) + krow * D + col0);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
                 float4 a = dst[i];
@@ -316,7 +449,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 dst[i] = a;
               }
             } else {
-              uint4 *dst = reinterpret_cast<uint4 *>((which ? p.dk_out : p.dv_out) + krow * D + c * 32);
+              uint4 *dst = reinterpret_cast<uint4 *>((which ? p.dk_out : p.dv_out) + krow * D + col0);
 #pragma unroll
               for (int i = 0; i < 4; ++i)
                 dst[i] = make_uint4(pack_bf16(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
@@ -330,6 +463,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       tc_fence_before();
       mbar_arrive(bar_acc_empty);
     }
+    if (lane == 0) bulk_wait0();  // all reduce-adds of this warp have been performed
   }
 
   __syncwarp();
@@ -339,28 +473,32 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+  if (warp == 9) { tc_fence_after(); tmem_dealloc(tmem, 512); }
 }
 
-// delta[h, tok] = sum_d dO * O  and  lse2 = lse * log2(e); one warp per (token, head).
+// Row statistics of the backward pass, stored per 128-row query tile:
+// stats[head][tile][0][i] = lse * log2(e) (+inf for rows past the tile's end),
+// stats[head][tile][1][i] = scale * sum_d dO * O (0 past the end).  One warp per 16 rows.
 template <int D>
-__global__ void bwd_preprocess_kernel(const __nv_bfloat16 *o, const __nv_bfloat16 *d_o, const float *lse, float *delta,
-                                      float *lse2, long long n_tok, int h_q) {
-  const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (w >= n_tok * h_q) return;
-  const long long tok = w / h_q;
-  const int head = (int)(w % h_q);
+__global__ void bwd_preprocess_kernel(const __nv_bfloat16 *o, const __nv_bfloat16 *d_o, const float *lse, const int32_t *tiles,
+                                      float *stats, long long n_tok, long long n_tiles, int h_q, float scale) {
+  const int tile = blockIdx.x, head = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tok0 = tiles[2 * tile], rows = tiles[2 * tile + 1];
+  float *out = stats + ((long long)head * n_tiles + tile) * 256;
   constexpr int PER = D / 32;
-  const __nv_bfloat16 *po = o + w * D + lane * PER, *pd = d_o + w * D + lane * PER;
-  float acc = 0.f;
+  for (int i = warp; i < 128; i += 8) {
+    float acc = 0.f, l2 = INFINITY;
+    if (i < rows) {
+      const long long w = ((long long)tok0 + i) * h_q + head;
+      const __nv_bfloat16 *po = o + w * D + lane * PER, *pd = d_o + w * D + lane * PER;
 #pragma unroll
-  for (int i = 0; i < PER; ++i) acc += __bfloat162float(po[i]) * __bfloat162float(pd[i]);
+      for (int e = 0; e < PER; ++e) acc += __bfloat162float(po[e]) * __bfloat162float(pd[e]);
 #pragma unroll
-  for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-  if (lane == 0) {
-    delta[(long long)head * n_tok + tok] = acc;
-    lse2[(long long)head * n_tok + tok] = lse[(long long)head * n_tok + tok] * 1.4426950408889634f;
+      for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+      l2 = lse[(long long)head * n_tok + tok0 + i] * 1.4426950408889634f;
+    }
+    if (lane == 0) { out[i] = l2; out[128 + i] = acc * scale; }
   }
 }
 

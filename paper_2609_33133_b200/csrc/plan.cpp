@@ -104,9 +104,15 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
   const int ng = p->n_groups;
 
   // q-segment tables for the backward kernels
-  p->seg_replay.clear(); p->seg_prefill.clear();
-  for (int i = 0; i < (int)nb; ++i) { p->seg_replay.push_back(p->cu_r[i]); p->seg_replay.push_back(p->branch_len[i]); }
-  for (int g = 0; g < ng; ++g) { p->seg_prefill.push_back(p->cu_p[g]); p->seg_prefill.push_back(p->prompt_len[g]); }
+  // (a segment's 128-row query tiles are numbered consecutively; the per-row
+  // statistics of the backward pass are stored tile by tile in that numbering)
+  p->seg_replay.clear(); p->seg_prefill.clear(); p->tiles_replay.clear(); p->tiles_prefill.clear();
+  auto add_segment = [](std::vector<int32_t> &segs, std::vector<int32_t> &tiles, int tok0, int len) {
+    segs.push_back(tok0); segs.push_back(len); segs.push_back((int32_t)(tiles.size() / 2));
+    for (int t = 0; t < cdiv(len, kTileQ); ++t) { tiles.push_back(tok0 + t * kTileQ); tiles.push_back(std::min(kTileQ, len - t * kTileQ)); }
+  };
+  for (int i = 0; i < (int)nb; ++i) add_segment(p->seg_replay, p->tiles_replay, p->cu_r[i], p->branch_len[i]);
+  for (int g = 0; g < ng; ++g) add_segment(p->seg_prefill, p->tiles_prefill, p->cu_p[g], p->prompt_len[g]);
 
   // prompt-KV shards per group: shard = a run of whole KV tiles
   p->group_splits.resize(ng);
@@ -200,8 +206,9 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
   if (p->max_splits > 1)
     p->ws_fwd = al((size_t)p->max_splits * (size_t)tr * hq * dd * 4) + al((size_t)p->max_splits * (size_t)tr * hq * 4);
   const size_t tmax = (size_t)std::max<int64_t>(tp, tr);
-  // backward: dq accumulator fp32 [tokens,H_q,d], delta and scaled lse [H_q,tokens] fp32
-  p->ws_bwd = al(tmax * hq * dd * 4) + 2 * al(tmax * hq * 4);
+  // backward: dq accumulator fp32 [tokens,H_q,d]; row statistics [H_q][tiles][2][128] fp32
+  const size_t ntile = std::max(p->tiles_replay.size(), p->tiles_prefill.size()) / 2;
+  p->ws_bwd = al(tmax * hq * dd * 4) + al(hq * ntile * 2 * kTileQ * 4);
   return AUGTREE_OK;
 }
 

@@ -41,10 +41,12 @@ struct augtree_plan {
   int64_t total_p = 0, total_r = 0;
   std::vector<int32_t> prompt_len, n_br, branch_len;
   std::vector<int32_t> cu_p, cu_b, cu_r, branch_group, group_splits;
-  std::vector<int32_t> seg_replay, seg_prefill;
+  std::vector<int32_t> seg_replay, seg_prefill;    // [n][3] {first query token, length, first tile index}
+  std::vector<int32_t> tiles_replay, tiles_prefill;  // [n_tiles][2] {first token, rows}: 128-row query tiles per segment
   augtree::Sched sched[augtree::SCHED_COUNT];
   int32_t *d_seg_replay = nullptr, *d_seg_prefill = nullptr, *d_branch_group = nullptr, *d_group_splits = nullptr;
   int32_t *d_cu_r = nullptr;
+  int32_t *d_tiles_replay = nullptr, *d_tiles_prefill = nullptr;
   int *d_status = nullptr;  // [2]: status, detail
   augtree::Timing *timing = nullptr;  // optional CUDA-event timing of the tile kernels
   size_t ws_fwd = 0, ws_bwd = 0;

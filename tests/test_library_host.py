@@ -72,8 +72,8 @@ def test_tables_bit_exact(binding, pl, bl, hq, hkv, lanes, splits):
     assert (plan.metadata(B.TBL_CU_BRANCH) == ref["cu_b"]).all()
     assert (plan.metadata(B.TBL_CU_RESPONSE) == ref["cu_r"]).all()
     assert (plan.metadata(B.TBL_GROUP_SPLITS) == ref["group_splits"]).all()
-    assert (plan.metadata(B.TBL_REPLAY_SEGMENTS).reshape(-1, 2) == ref["seg_replay"]).all()
-    assert (plan.metadata(B.TBL_PREFILL_SEGMENTS).reshape(-1, 2) == ref["seg_prefill"]).all()
+    assert (plan.metadata(B.TBL_REPLAY_SEGMENTS).reshape(-1, 3) == ref["seg_replay"]).all()
+    assert (plan.metadata(B.TBL_PREFILL_SEGMENTS).reshape(-1, 3) == ref["seg_prefill"]).all()
     for base, key, w, wf in [(B.TBL_PREFILL_FWD_ITEMS, "prefill_fwd", 12, 10), (B.TBL_REPLAY_FWD_ITEMS, "replay_fwd", 12, 10),
                              (B.TBL_REPLAY_BWD_ITEMS, "replay_bwd", 8, 7), (B.TBL_PREFILL_BWD_ITEMS, "prefill_bwd", 8, 7)]:
         items = plan.metadata(base).reshape(-1, w)
