@@ -49,9 +49,12 @@ def pair_counts(w):
 def useful_flops(w):
     pre, rep, flat = pair_counts(w)
     per_pair = 14 * w.head_dim * w.h_q
-    return {"total": per_pair * (pre + rep), "prefill_fwd": 4 * w.head_dim * w.h_q * pre, "replay_fwd": 4 * w.head_dim * w.h_q * rep,
-            "replay_bwd": 10 * w.head_dim * w.h_q * rep, "prefill_bwd": 10 * w.head_dim * w.h_q * pre,
-            "flattened_total": per_pair * flat, "reuse_factor": flat / (pre + rep)}
+    dh = w.head_dim * w.h_q
+    # per kernel: the FLOPs its GEMMs execute (the two backward kernels both recompute S and dP:
+    # 4 + 3 GEMMs for the 5 of the textbook backward; `total` counts the 5)
+    return {"total": per_pair * (pre + rep), "prefill_fwd": 4 * dh * pre, "replay_fwd": 4 * dh * rep,
+            "replay_bwd_dkdv": 8 * dh * rep, "prefill_bwd_dkdv": 8 * dh * pre, "replay_bwd_dq": 6 * dh * rep,
+            "prefill_bwd_dq": 6 * dh * pre, "flattened_total": per_pair * flat, "reuse_factor": flat / (pre + rep)}
 
 
 def peaks():
@@ -247,19 +250,21 @@ def main():
     st = plan.device_status()
     if st != (0, 0):
         raise RuntimeError(f"device status {st}")
-    kt = [plan.kernel_time(k) for k in range(4)]
+    kt = [plan.kernel_time(k) for k in range(6)]
     plan.set_timing(False)
     ms_step = ms / args.steps
     value = world * fl["total"] / (ms_step * 1e-3) / 1e12
 
     # dominant kernel: the replay backward tile kernel
-    names = ["prefill_fwd", "replay_fwd", "replay_bwd", "prefill_bwd"]
+    names = ["prefill_fwd", "replay_fwd", "replay_bwd_dkdv", "prefill_bwd_dkdv", "replay_bwd_dq", "prefill_bwd_dq"]
+    kfun = {"prefill_fwd": "fwd_kernel", "replay_fwd": "fwd_kernel", "replay_bwd_dkdv": "bwd_kernel", "prefill_bwd_dkdv": "bwd_kernel",
+            "replay_bwd_dq": "dq_kernel", "prefill_bwd_dq": "dq_kernel"}
     per_kernel = {}
     for n, (tot, cnt) in zip(names, kt):
         if cnt:
             per_kernel[n] = {"ms": tot / cnt, "tflops": fl[n] / (tot / cnt * 1e-3) / 1e12, "launches": cnt}
     dom = max(per_kernel, key=lambda n: per_kernel[n]["ms"])
-    roofline = {"bound": "tensor", "kernel": f"{'bwd' if 'bwd' in dom else 'fwd'}_kernel ({dom})", "achieved": per_kernel[dom]["tflops"],
+    roofline = {"bound": "tensor", "kernel": f"{kfun[dom]} ({dom})", "achieved": per_kernel[dom]["tflops"],
                 "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": per_kernel[dom]["tflops"] / pk["bf16_tflops"],
                 "peak_source": f"{pk['source']} cuBLAS bf16 burst", "traffic": None}
 

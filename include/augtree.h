@@ -92,7 +92,9 @@ enum {
   AUGTREE_TBL_REPLAY_SEGMENTS = 15,  /* [n_branches][3] {first response token, length, first query-tile index} */
   AUGTREE_TBL_PREFILL_SEGMENTS = 16, /* [n_groups][3]   {first prompt token, length, first query-tile index}   */
   AUGTREE_TBL_GROUP_SPLITS = 17,     /* [n_groups] prompt-KV shards actually used           */
-  AUGTREE_TBL_COUNT = 18
+  AUGTREE_TBL_REPLAY_DQ_ITEMS = 18,  AUGTREE_TBL_REPLAY_DQ_LANE_PTR = 19,  AUGTREE_TBL_REPLAY_DQ_ORDER = 20,
+  AUGTREE_TBL_PREFILL_DQ_ITEMS = 21, AUGTREE_TBL_PREFILL_DQ_LANE_PTR = 22, AUGTREE_TBL_PREFILL_DQ_ORDER = 23,
+  AUGTREE_TBL_COUNT = 24
 };
 #define AUGTREE_FWD_ITEM_INTS 12
 #define AUGTREE_BWD_ITEM_INTS 8
@@ -127,6 +129,10 @@ int augtree_plan_workspace_bytes(const augtree_plan_t *plan, size_t *fwd_bytes, 
  *   backward item [8] : kv_tok0, kv_pos0, kv_rows, kv_head, mode, seg0, nseg,
  *                       weight;  mode 0 = causal inside one sequence, mode 1 =
  *     shared prompt keys against every response query of the group (Eq. 2).
+ *     These are the units of the key-side backward kernel (dK, dV).
+ *   dQ item [12]: a forward item that is never sharded; field 8 holds the
+ *     index of the query tile (segment's first tile index + tile) instead of
+ *     the shard number.  Units of the query-side backward kernel.
  *   *_LANE_PTR [n_lanes+1], *_ORDER [n_items]: lane l runs the items
  *     ORDER[LANE_PTR[l] .. LANE_PTR[l+1]) in that order.
  */
@@ -160,8 +166,9 @@ int augtree_replay_fwd(const augtree_plan_t *plan, const void *q_r, const void *
  * gradients of all branches and query heads are ADDED into the fp32
  * accumulators dkp_acc, dvp_acc [sumP,H_kv,d], which the caller zeroes first
  * (or sets AUGTREE_FLAG_ZERO_PROMPT_GRAD in the descriptor).  Each prompt-KV
- * tile is owned by one lane, so this sum has a fixed order; dq_r is summed
- * with fp32 atomics in scratch and rounded once.
+ * tile is owned by one lane, so this sum has a fixed order; dq_r comes from a
+ * second, query-stationary kernel in which each query tile has one owner.
+ * No atomics are used: results are bitwise repeatable.
  */
 int augtree_replay_bwd(const augtree_plan_t *plan, const void *q_r, const void *k_r, const void *v_r,
                        const void *k_p, const void *v_p, const void *o_r, const float *lse_r,
@@ -232,7 +239,8 @@ int augtree_last_device_status(const augtree_plan_t *plan, int *status, int *det
  * each call resets the record.  The events are created on the first call,
  * which is therefore not free; the launches themselves stay asynchronous.
  * augtree_get_kernel_time waits for the recorded launches of one kernel
- * (0 prefill fwd, 1 replay fwd, 2 replay bwd, 3 prefill bwd) and returns their
+ * (0 prefill fwd, 1 replay fwd, 2 replay bwd dK/dV, 3 prefill bwd dK/dV, 4 replay bwd dQ,
+ * 5 prefill bwd dQ) and returns their
  * summed device time and count.
  */
 int augtree_set_timing(augtree_plan_t *plan, int enable);

@@ -39,7 +39,9 @@ def build_tables(prompt_len, branch_len, h_q, h_kv, kv_splits=1):
     flat = [r for b in branch_len for r in b]
     cu_r = prefix(flat)
     kv_splits = max(1, kv_splits)
-    pf, rf, rb, pb, gsplits = [], [], [], [], []
+    pf, rf, rb, pb, gsplits, rq, pq = [], [], [], [], [], [], []
+    ptile0 = prefix([_cdiv(x, TQ) for x in prompt_len])
+    rtile0 = prefix([_cdiv(x, TQ) for x in flat])
     for g, P in enumerate(prompt_len):
         p0 = cu_p[g]
         na = _cdiv(P, TK)
@@ -52,11 +54,15 @@ def build_tables(prompt_len, branch_len, h_q, h_kv, kv_splits=1):
                 vis = t * TQ + rows
                 for j in range(rep):
                     pf.append([p0 + t * TQ, t * TQ, rows, c * rep + j, 0, 0, p0, vis, 0, 1, _cdiv(vis, TK), c])
+                    pq.append([p0 + t * TQ, t * TQ, rows, c * rep + j, 0, 0, p0, vis, ptile0[g] + t, 1, _cdiv(vis, TK), c])
             for bi in range(cu_b[g], cu_b[g + 1]):
                 R, r0 = flat[bi], cu_r[bi]
                 for t in range(_cdiv(R, TQ)):
                     rows = min(TQ, R - t * TQ)
                     vis = t * TQ + rows
+                    for j in range(rep):
+                        rq.append([r0 + t * TQ, t * TQ, rows, c * rep + j, p0, P, r0, vis, rtile0[bi] + t, 1,
+                                   _cdiv(P, TK) + _cdiv(vis, TK), c])
                     for j in range(rep):
                         for s in range(ns):
                             a0 = s * shard_tiles * TK
@@ -79,6 +85,7 @@ def build_tables(prompt_len, branch_len, h_q, h_kv, kv_splits=1):
     return {
         "cu_p": np.asarray(cu_p, np.int32), "cu_b": np.asarray(cu_b, np.int32), "cu_r": np.asarray(cu_r, np.int32),
         "prefill_fwd": arr(pf, 12), "replay_fwd": arr(rf, 12), "replay_bwd": arr(rb, 8), "prefill_bwd": arr(pb, 8),
+        "replay_dq": arr(rq, 12), "prefill_dq": arr(pq, 12),
         "group_splits": np.asarray(gsplits, np.int32),
         # segments: first token, length, index of the segment's first 128-row query tile
         "seg_replay": np.asarray([[cu_r[i], flat[i], sum(_cdiv(x, TQ) for x in flat[:i])] for i in range(len(flat))],

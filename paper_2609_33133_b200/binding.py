@@ -25,7 +25,8 @@ FWD_ITEM_INTS, BWD_ITEM_INTS = 12, 8
 (TBL_CU_PROMPT, TBL_CU_BRANCH, TBL_CU_RESPONSE, TBL_PREFILL_FWD_ITEMS, TBL_PREFILL_FWD_LANE_PTR, TBL_PREFILL_FWD_ORDER,
  TBL_REPLAY_FWD_ITEMS, TBL_REPLAY_FWD_LANE_PTR, TBL_REPLAY_FWD_ORDER, TBL_REPLAY_BWD_ITEMS, TBL_REPLAY_BWD_LANE_PTR,
  TBL_REPLAY_BWD_ORDER, TBL_PREFILL_BWD_ITEMS, TBL_PREFILL_BWD_LANE_PTR, TBL_PREFILL_BWD_ORDER, TBL_REPLAY_SEGMENTS,
- TBL_PREFILL_SEGMENTS, TBL_GROUP_SPLITS) = range(18)
+ TBL_PREFILL_SEGMENTS, TBL_GROUP_SPLITS, TBL_REPLAY_DQ_ITEMS, TBL_REPLAY_DQ_LANE_PTR, TBL_REPLAY_DQ_ORDER,
+ TBL_PREFILL_DQ_ITEMS, TBL_PREFILL_DQ_LANE_PTR, TBL_PREFILL_DQ_ORDER) = range(24)
 
 EXPORTS = ["augtree_plan_create", "augtree_plan_destroy", "augtree_plan_workspace_bytes", "augtree_plan_metadata",
            "augtree_prefill_fwd", "augtree_replay_fwd", "augtree_replay_bwd", "augtree_prefill_bwd",

@@ -8,6 +8,7 @@
 #include <new>
 
 #include "bwd_kernel.cuh"
+#include "dq_kernel.cuh"
 #include "fwd_kernel.cuh"
 #include "plan.h"
 
@@ -56,21 +57,6 @@ int make_map(CUtensorMap *m, const void *ptr, long long tokens, int heads, int d
   const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? AUGTREE_OK : AUGTREE_ERR_CUDA;
-}
-
-// Tensor map over the fp32 dQ accumulator [tokens, heads, d]: boxes of 32 tokens
-// by 32 floats (128 bytes) of one head, 128-byte swizzle, used for reduce-adds.
-int make_map_f32(CUtensorMap *m, void *ptr, long long tokens, int heads, int d) {
-  EncodeTiledFn enc = get_encode();
-  if (!enc) return AUGTREE_ERR_CUDA;
-  if (tokens < 1) tokens = 1;
-  const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)heads, (cuuint64_t)tokens};
-  const cuuint64_t strides[2] = {(cuuint64_t)d * 4, (cuuint64_t)heads * d * 4};
-  const cuuint32_t box[3] = {32, 1, 32};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? AUGTREE_OK : AUGTREE_ERR_CUDA;
 }
 
@@ -140,35 +126,31 @@ struct BwdArgs {
   const int32_t *d_segs;
   const int32_t *d_tiles;  // [n_tiles][2] query tiles of the call's query tensor
   long long n_tiles;
+  const Sched *dq_sched;   // query-side units
+  // key ranges of the query-side kernel: unmasked range tensor (a), causal range tensor (b)
+  const void *ka, *va; long long a_tok;
 };
 
+// One backward call: row statistics, then the key-side kernel (dK, dV), then the query-side kernel (dQ).
 template <int D>
 int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *ws, cudaStream_t st) {
-  const size_t hq = pl->h_q;
-  const size_t n_el = (size_t)a.q_tok * hq * D;
-  if (n_el == 0) return AUGTREE_OK;
-  uint8_t *w = static_cast<uint8_t *>(ws);
-  float *dq_acc = reinterpret_cast<float *>(w);
-  // region sizes must match build_plan_host: sized for max(total_p, total_r)
-  const size_t tmax = (size_t)(pl->total_p > pl->total_r ? pl->total_p : pl->total_r);
-  float *stats = reinterpret_cast<float *>(w + al256(tmax * hq * D * 4));
-  if (cudaMemsetAsync(dq_acc, 0, n_el * 4, st) != cudaSuccess) return AUGTREE_ERR_CUDA;
+  if (a.q_tok == 0) return AUGTREE_OK;
+  float *stats = static_cast<float *>(ws);
   {
     const dim3 grid((unsigned)a.n_tiles, (unsigned)pl->h_q);
     bwd_preprocess_kernel<D><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(a.o), static_cast<const __nv_bfloat16 *>(a.d_o),
                                                    a.lse, a.d_tiles, stats, a.q_tok, a.n_tiles, pl->h_q, pl->scale);
     ++g_launches;
   }
+  CUtensorMap mq, mdo, mk0, mv0, mk1, mv1;
+  int r;
+  if ((r = make_map(&mq, a.q, a.q_tok, pl->h_q, D))) return r;
+  if ((r = make_map(&mdo, a.d_o, a.q_tok, pl->h_q, D))) return r;
+  if ((r = make_map(&mk0, a.k0, a.kv0_tok, pl->h_kv, D))) return r;
+  if ((r = make_map(&mv0, a.v0, a.kv0_tok, pl->h_kv, D))) return r;
+  if ((r = make_map(&mk1, a.k1, a.kv1_tok, pl->h_kv, D))) return r;
+  if ((r = make_map(&mv1, a.v1, a.kv1_tok, pl->h_kv, D))) return r;
   if (s.n_items() > 0) {
-    CUtensorMap mq, mdo, mk0, mv0, mk1, mv1, mdq;
-    int r;
-    if ((r = make_map(&mq, a.q, a.q_tok, pl->h_q, D))) return r;
-    if ((r = make_map(&mdo, a.d_o, a.q_tok, pl->h_q, D))) return r;
-    if ((r = make_map(&mk0, a.k0, a.kv0_tok, pl->h_kv, D))) return r;
-    if ((r = make_map(&mv0, a.v0, a.kv0_tok, pl->h_kv, D))) return r;
-    if ((r = make_map(&mk1, a.k1, a.kv1_tok, pl->h_kv, D))) return r;
-    if ((r = make_map(&mv1, a.v1, a.kv1_tok, pl->h_kv, D))) return r;
-    if ((r = make_map_f32(&mdq, dq_acc, a.q_tok, pl->h_q, D))) return r;
     BwdParams p;
     p.items = s.d_items; p.lane_ptr = s.d_lane_ptr; p.segs = a.d_segs; p.stats = stats;
     p.dk_out = static_cast<__nv_bfloat16 *>(a.dk_out); p.dv_out = static_cast<__nv_bfloat16 *>(a.dv_out);
@@ -183,14 +165,30 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     }
     const int kind = (int)(&s - pl->sched);
     timing_mark(pl, kind, false, st);
-    bwd_kernel<D><<<pl->n_lanes, kBwdThreads, BwdSmem<D>::kBytes, st>>>(mq, mdo, mk0, mv0, mk1, mv1, mdq, p);
+    bwd_kernel<D><<<pl->n_lanes, kBwdThreads, BwdSmem<D>::kBytes, st>>>(mq, mdo, mk0, mv0, mk1, mv1, p);
     timing_mark(pl, kind, true, st);
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return AUGTREE_ERR_CUDA;
   }
-  {
-    const long long n4 = (long long)(n_el / 4);
-    cast_bf16_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(dq_acc, static_cast<__nv_bfloat16 *>(a.dq), n4);
+  if (a.dq_sched->n_items() > 0) {
+    CUtensorMap mka, mva;
+    if ((r = make_map(&mka, a.ka, a.a_tok, pl->h_kv, D))) return r;
+    if ((r = make_map(&mva, a.va, a.a_tok, pl->h_kv, D))) return r;
+    DqParams p;
+    p.items = a.dq_sched->d_items; p.lane_ptr = a.dq_sched->d_lane_ptr; p.stats = stats;
+    p.dq = static_cast<__nv_bfloat16 *>(a.dq); p.n_tiles = a.n_tiles; p.h_q = pl->h_q;
+    p.scale = pl->scale; p.scale_log2 = pl->scale * 1.4426950408889634f; p.status = pl->d_status;
+    static bool attr_set[2] = {false, false};
+    if (!attr_set[D / 128]) {
+      if (cudaFuncSetAttribute(dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<D>::kBytes) != cudaSuccess)
+        return AUGTREE_ERR_CUDA;
+      attr_set[D / 128] = true;
+    }
+    const int kind = (int)(a.dq_sched - pl->sched);
+    timing_mark(pl, kind, false, st);
+    // causal keys come from the queries' own sequence tensor (k0/v0)
+    dq_kernel<D><<<pl->n_lanes, kDqThreads, DqSmem<D>::kBytes, st>>>(mq, mdo, mka, mva, mk0, mv0, p);
+    timing_mark(pl, kind, true, st);
     ++g_launches;
   }
   return cudaGetLastError() == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
@@ -306,6 +304,10 @@ int augtree_plan_metadata(const augtree_plan_t *pl, int table_id, void *host_dst
         const Sched &s = pl->sched[(table_id - 3) / 3];
         const int which = (table_id - 3) % 3;
         v = which == 0 ? &s.items : which == 1 ? &s.lane_ptr : &s.order;
+      } else if (table_id >= AUGTREE_TBL_REPLAY_DQ_ITEMS && table_id <= AUGTREE_TBL_PREFILL_DQ_ORDER) {
+        const Sched &s = pl->sched[SCHED_REPLAY_DQ + (table_id - AUGTREE_TBL_REPLAY_DQ_ITEMS) / 3];
+        const int which = (table_id - AUGTREE_TBL_REPLAY_DQ_ITEMS) % 3;
+        v = which == 0 ? &s.items : which == 1 ? &s.lane_ptr : &s.order;
       }
   }
   if (!v) return AUGTREE_ERR_INVALID_ARG;
@@ -418,6 +420,7 @@ int augtree_replay_bwd(const augtree_plan_t *pl, const void *q_r, const void *k_
   a.k0 = k_r; a.v0 = v_r; a.kv0_tok = pl->total_r; a.k1 = k_p; a.v1 = v_p; a.kv1_tok = pl->total_p;
   a.dq = dq_r; a.dk_out = dk_r; a.dv_out = dv_r; a.dk_acc = dkp_acc; a.dv_acc = dvp_acc; a.causal_fp32 = 0;
   a.d_segs = pl->d_seg_replay; a.d_tiles = pl->d_tiles_replay; a.n_tiles = (long long)pl->tiles_replay.size() / 2;
+  a.dq_sched = &pl->sched[SCHED_REPLAY_DQ]; a.ka = k_p; a.va = v_p; a.a_tok = pl->total_p;
   const Sched &s = pl->sched[SCHED_REPLAY_BWD];
   return pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, st) : launch_bwd<64>(pl, s, a, ws, st);
 }
@@ -438,6 +441,7 @@ int augtree_prefill_bwd(const augtree_plan_t *pl, const void *q_p, const void *k
   a.k0 = k_p; a.v0 = v_p; a.kv0_tok = pl->total_p; a.k1 = k_p; a.v1 = v_p; a.kv1_tok = pl->total_p;
   a.dq = dq_p; a.dk_out = nullptr; a.dv_out = nullptr; a.dk_acc = dkp_acc; a.dv_acc = dvp_acc; a.causal_fp32 = 1;
   a.d_segs = pl->d_seg_prefill; a.d_tiles = pl->d_tiles_prefill; a.n_tiles = (long long)pl->tiles_prefill.size() / 2;
+  a.dq_sched = &pl->sched[SCHED_PREFILL_DQ]; a.ka = k_p; a.va = v_p; a.a_tok = pl->total_p;
   const Sched &s = pl->sched[SCHED_PREFILL_BWD];
   r = pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, st) : launch_bwd<64>(pl, s, a, ws, st);
   if (r) return r;

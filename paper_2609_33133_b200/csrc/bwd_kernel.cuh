@@ -1,27 +1,26 @@
-// Backward tile kernel, KV-stationary: one persistent CTA per replay lane walks
-// its list of (KV tile, KV head) items.  An item keeps its K and V tile in
+// Backward, key side (dK, dV), KV-stationary: one persistent CTA per replay lane
+// walks its list of (KV tile, KV head) items.  An item keeps its K and V tile in
 // shared memory and streams past it every query tile that can see it: for a
-// prompt-KV tile in replay, all response tiles of all G branches and all
-// query heads of the KV head, which is the many-to-one sum of Eq. 2 done in
-// one TMEM accumulator in a fixed order; for a tile inside a sequence, the
-// causal query tiles of that sequence.
+// prompt-KV tile in replay, all response tiles of all G branches and all query
+// heads of the KV head, which is the many-to-one sum of Eq. 2 done in one TMEM
+// accumulator in a fixed order by one owner; for a tile inside a sequence, the
+// causal query tiles of that sequence.  (The query side, dQ, is computed by
+// dq_kernel, query-stationary, so that neither side needs atomics.)
 //
 // Per (KV tile, Q tile, head) pair T, with S^T = K Q^T so that a TMEM lane is a key:
 //   P^T  = exp2(S^T * scale*log2e - lse2[q])          (element-wise warps)
 //   dP^T = V dO^T
 //   dS^T = P^T * (scale*dP^T - scale*delta[q])        (element-wise warps)
 //   dV  += P^T dO      (A = P^T from TMEM)
-//   dK  += dS^T Q      (A = dS^T from shared memory, K-major)
-//   dQ   = dS K        (A = the same dS^T tile read MN-major) -> fp32 TMA reduce-add
+//   dK  += dS^T Q      (A = dS^T from TMEM)
 //
 // Warp roles (320 threads): warps 0-7 element-wise (warp w: TMEM lanes
 // 32*(w%4).., query columns 64*(w/4)..), warp 8 lane 0 TMA loads, warp 9 lane 0
 // MMA issue.  TMEM columns: R0 [0,128) S^T, overwritten in place by P^T (bf16);
-// R1 [128,256) dP^T, later dQ; dV at 256; dK at 256 + D.
-//
-// MMA issue order in steady state: dP(T), S(T+1), dK(T), dQ(T), dV(T+1), so the
-// tensor pipe has independent work while the warps turn S into P, dP into dS
-// and drain dQ.
+// R1 [128,256) dP^T, overwritten in place by dS^T (bf16); dV at 256; dK at 256 + D.
+// MMA issue order in steady state: dP(T), dV(T), S(T+1), dK(T); the tensor pipe
+// executes in order, so S(T+1) may overwrite R0 once dV(T) is issued and
+// dP(T+1) may overwrite R1 once dK(T) is issued.
 #pragma once
 #include <cuda.h>
 
@@ -44,18 +43,16 @@ struct BwdParams {
 };
 
 constexpr int kBwdThreads = 320;
-constexpr int kBwdStages = 2;
 
 template <int D>
 struct BwdSmem {
+  static constexpr int kStages = 2;
   static constexpr int kTileBytes = 128 * D * 2;
-  static constexpr int kDsBytes = 128 * 128 * 2;
   static constexpr int kOffK = 0, kOffV = kTileBytes;
-  static constexpr int kOffQ = 2 * kTileBytes;                        // [kBwdStages]
-  static constexpr int kOffDo = kOffQ + kBwdStages * kTileBytes;      // [kBwdStages]
-  static constexpr int kOffDs = kOffDo + kBwdStages * kTileBytes;     // dS^T tile, reused as dQ staging
-  static constexpr int kOffStats = kOffDs + kDsBytes;                 // [kBwdStages][2][128] floats
-  static constexpr int kOffBar = kOffStats + kBwdStages * 1024;
+  static constexpr int kOffQ = 2 * kTileBytes;                     // [kStages]
+  static constexpr int kOffDo = kOffQ + kStages * kTileBytes;      // [kStages]
+  static constexpr int kOffStats = kOffDo + kStages * kTileBytes;  // [kStages][2][128] floats
+  static constexpr int kOffBar = kOffStats + kStages * 1024;
   static constexpr int kBytes = kOffBar + 256;
 };
 
@@ -64,24 +61,16 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-// fp32 reduce-add of a shared-memory box into a global tensor
-__device__ __forceinline__ void tma_reduce_add_3d(const void *tmap, uint32_t src, int c0, int c1, int c2) {
-  asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
-               ::"l"(tmap), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
            const __grid_constant__ CUtensorMap tm_k0, const __grid_constant__ CUtensorMap tm_v0,
-           const __grid_constant__ CUtensorMap tm_k1, const __grid_constant__ CUtensorMap tm_v1,
-           const __grid_constant__ CUtensorMap tm_dq, const BwdParams p) {
+           const __grid_constant__ CUtensorMap tm_k1, const __grid_constant__ CUtensorMap tm_v1, const BwdParams p) {
   using SM = BwdSmem<D>;
   constexpr int TILE = SM::kTileBytes;
   constexpr int NBOX = D / 64;
+  constexpr int NST = SM::kStages;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   if (base & 1023u) {  // the 128-byte swizzle needs 1024-byte aligned tiles
@@ -89,26 +78,24 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     return;
   }
   const uint32_t sK = base + SM::kOffK, sV = base + SM::kOffV, sQ0 = base + SM::kOffQ, sDo0 = base + SM::kOffDo;
-  const uint32_t sDs = base + SM::kOffDs, sStats0 = base + SM::kOffStats;
+  const uint32_t sStats0 = base + SM::kOffStats;
   const uint32_t bars = base + SM::kOffBar;
   const uint32_t bar_kv_full = bars, bar_kv_empty = bars + 8;
-  const uint32_t bar_q_full = bars + 16, bar_q_empty = bars + 32;    // [2] each
-  const uint32_t bar_do_full = bars + 48, bar_do_empty = bars + 64;  // [2] each
-  const uint32_t bar_s_full = bars + 80, bar_p_ready = bars + 88, bar_dp_full = bars + 96, bar_ds_ready = bars + 104;
-  const uint32_t bar_dq_full = bars + 112, bar_drained = bars + 120, bar_stage_free = bars + 128;
-  const uint32_t bar_acc_full = bars + 136, bar_acc_empty = bars + 144;
-  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_raw + SM::kOffBar + 160);
-  volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + SM::kOffBar + 168);
+  const uint32_t bar_q_full = bars + 16, bar_q_empty = bars + 48;     // [NST <= 4] each
+  const uint32_t bar_do_full = bars + 80, bar_do_empty = bars + 112;  // [NST <= 4] each
+  const uint32_t bar_s_full = bars + 144, bar_p_ready = bars + 152, bar_dp_full = bars + 160, bar_ds_ready = bars + 168;
+  const uint32_t bar_acc_full = bars + 176, bar_acc_empty = bars + 184;
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_raw + SM::kOffBar + 192);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + SM::kOffBar + 200);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     mbar_init(bar_kv_full, 1); mbar_init(bar_kv_empty, 1);
-    for (int s = 0; s < kBwdStages; ++s) {
+    for (int s = 0; s < NST; ++s) {
       mbar_init(bar_q_full + 8 * s, 1); mbar_init(bar_q_empty + 8 * s, 1);
       mbar_init(bar_do_full + 8 * s, 1); mbar_init(bar_do_empty + 8 * s, 1);
     }
     mbar_init(bar_s_full, 1); mbar_init(bar_p_ready, 256); mbar_init(bar_dp_full, 1); mbar_init(bar_ds_ready, 256);
-    mbar_init(bar_dq_full, 1); mbar_init(bar_drained, 256); mbar_init(bar_stage_free, 8);
     mbar_init(bar_acc_full, 1); mbar_init(bar_acc_empty, 256);
     *abort_flag = 0;
     fence_barrier_init();
@@ -147,7 +134,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           const int nqt = (s_len + 127) >> 7;
           for (int qt = mode ? 0 : (kv_pos0 >> 7); qt < nqt && ok; ++qt)
             for (int j = 0; j < rep; ++j, ++T) {
-              const uint32_t st = T % kBwdStages, par = ((T / kBwdStages) & 1) ^ 1;
+              const uint32_t st = T % NST, par = ((T / NST) & 1) ^ 1;
               const int head = kvh * rep + j, row = s_tok0 + qt * 128;
               ok = mbar_wait(bar_q_empty + 8 * st, par, ab, WAIT_BWD_QDO_EMPTY);
               if (!ok) break;
@@ -167,34 +154,18 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       constexpr uint32_t IDESC_ST = make_idesc(128, 128, 0, 0);  // S^T, dP^T: both operands K-major
-      constexpr uint32_t IDESC_DV = make_idesc(128, D, 0, 1);    // dV: A = P^T (TMEM), B = dO MN-major
-      constexpr uint32_t IDESC_DK = make_idesc(128, D, 0, 1);    // dK: A = dS^T K-major (shared), B = Q MN-major
-      constexpr uint32_t IDESC_DQ = make_idesc(128, D, 1, 1);    // dQ: A = dS^T read MN-major, B = K MN-major
+      constexpr uint32_t IDESC_ACC = make_idesc(128, D, 0, 1);   // dV, dK: A from TMEM, B = dO / Q MN-major
       uint32_t ic = 0, T = 0;
       bool ok = true;
+      const uint32_t kk_lo = sdesc_lo(sK, 16), vk_lo = sdesc_lo(sV, 16);
       auto issue_s = [&](uint32_t Tn) -> bool {  // S^T(Tn) = K Q^T -> R0
-        const uint32_t st = Tn % kBwdStages;
-        if (!mbar_wait(bar_q_full + 8 * st, (Tn / kBwdStages) & 1, ab, WAIT_BWD_QDO_FULL)) return false;
+        const uint32_t st = Tn % NST;
+        if (!mbar_wait(bar_q_full + 8 * st, (Tn / NST) & 1, ab, WAIT_BWD_QDO_FULL)) return false;
         tc_fence_after();
-        const uint32_t sQ = sQ0 + st * TILE;
+        const uint32_t qk_lo = sdesc_lo(sQ0 + st * TILE, 16);
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-          mma_ss(tR0, make_sdesc(sK + off, 16, 1024), make_sdesc(sQ + off, 16, 1024), IDESC_ST, k > 0);
-        }
+        for (int k = 0; k < D / 16; ++k) mma_ss2(tR0, kk_lo + kstep_kmajor(k), qk_lo + kstep_kmajor(k), IDESC_ST, k > 0);
         tc_commit(bar_s_full);
-        return true;
-      };
-      auto issue_dv = [&](uint32_t Tn, uint32_t acc0) -> bool {  // dV += P^T(Tn) dO(Tn)
-        const uint32_t st = Tn % kBwdStages;
-        if (!mbar_wait(bar_p_ready, Tn & 1, ab, WAIT_BWD_PDS_FULL)) return false;
-        if (!mbar_wait(bar_do_full + 8 * st, (Tn / kBwdStages) & 1, ab, WAIT_BWD_QDO_FULL)) return false;
-        tc_fence_after();
-        const uint32_t sdO = sDo0 + st * TILE;
-#pragma unroll
-        for (int k = 0; k < 8; ++k)  // query columns 16k..16k+15: P^T sits at R0 columns 8k (k<4) or 64+8(k-4)
-          mma_ts(tDV, tR0 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), make_sdesc(sdO + k * 2048, 16384, 1024), IDESC_DV,
-                 acc0 | (uint32_t)(k > 0));
         return true;
       };
       for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
@@ -207,52 +178,44 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
         ok = mbar_wait(bar_kv_full, ic & 1, ab, WAIT_BWD_KV_FULL);
         if (!ok) break;
-        // prologue: S(T), dV(T) of the item's first pair
-        ok = issue_s(T);
-        if (!ok) break;
-        if (ic > 0) {
-          ok = mbar_wait(bar_acc_empty, (ic - 1) & 1, ab, WAIT_BWD_ACC_EMPTY);
-          if (!ok) break;
-        }
-        ok = issue_dv(T, 0u);
+        ok = issue_s(T);  // prologue: S^T of the item's first pair
         for (int i = 0; i < n_pairs && ok; ++i, ++T) {
-          const uint32_t st = T % kBwdStages;
-          const uint32_t sQ = sQ0 + st * TILE, sdO = sDo0 + st * TILE;
-          // dP^T(T) = V dO^T -> R1 (needs dQ(T-1) drained out of R1)
-          if (T > 0) {
-            ok = mbar_wait(bar_drained, (T - 1) & 1, ab, WAIT_BWD_DQ_FREE);
+          const uint32_t st = T % NST;
+          const uint32_t dok_lo = sdesc_lo(sDo0 + st * TILE, 16), dom_lo = sdesc_lo(sDo0 + st * TILE, 16384);
+          const uint32_t qm_lo = sdesc_lo(sQ0 + st * TILE, 16384);
+          const uint32_t acc0 = i > 0 ? 1u : 0u;
+          // ---- dP^T(T) = V dO^T -> R1
+          ok = mbar_wait(bar_do_full + 8 * st, (T / NST) & 1, ab, WAIT_BWD_QDO_FULL);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) mma_ss2(tR1, vk_lo + kstep_kmajor(k), dok_lo + kstep_kmajor(k), IDESC_ST, k > 0);
+          tc_commit(bar_dp_full);
+          // ---- dV += P^T(T) dO(T)
+          ok = mbar_wait(bar_p_ready, T & 1, ab, WAIT_BWD_PDS_FULL);
+          if (!ok) break;
+          if (i == 0 && ic > 0) {  // the previous item's dV/dK must have left TMEM
+            ok = mbar_wait(bar_acc_empty, (ic - 1) & 1, ab, WAIT_BWD_ACC_EMPTY);
             if (!ok) break;
           }
           tc_fence_after();
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-            mma_ss(tR1, make_sdesc(sV + off, 16, 1024), make_sdesc(sdO + off, 16, 1024), IDESC_ST, k > 0);
-          }
-          tc_commit(bar_dp_full);
-          tc_commit(bar_do_empty + 8 * st);  // dO(T) was last read by dV(T) (issued earlier) and dP(T)
-          // S^T(T+1)
+          for (int k = 0; k < 8; ++k)  // query columns 16k..16k+15: P^T sits at R0 columns 8k (k<4) or 64+8(k-4)
+            mma_ts2(tDV, tR0 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), dom_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
+          tc_commit(bar_do_empty + 8 * st);
+          // ---- S^T(T+1) (R0 is free: dV(T) was issued)
           if (i + 1 < n_pairs) {
             ok = issue_s(T + 1);
             if (!ok) break;
           }
-          // dK += dS^T(T) Q(T);  dQ(T) = dS(T) K -> R1
+          // ---- dK += dS^T(T) Q(T)
           ok = mbar_wait(bar_ds_ready, T & 1, ab, WAIT_BWD_PDS_FULL);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t acc0 = i > 0 ? 1u : 0u;
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {  // K dim = 128 queries: dS^T box k/4, 32 bytes per step
-            const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-            mma_ss(tDK, make_sdesc(sDs + off, 16, 1024), make_sdesc(sQ + k * 2048, 16384, 1024), IDESC_DK, acc0 | (uint32_t)(k > 0));
-          }
+          for (int k = 0; k < 8; ++k)
+            mma_ts2(tDK, tR1 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), qm_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
           tc_commit(bar_q_empty + 8 * st);
-#pragma unroll
-          for (int k = 0; k < 8; ++k)  // K dim = 128 keys: 16 rows of dS^T / K per step
-            mma_ss(tR1, make_sdesc(sDs + k * 2048, 16384, 1024), make_sdesc(sK + k * 2048, 16384, 1024), IDESC_DQ, k > 0);
-          tc_commit(bar_dq_full);
-          // dV += P^T(T+1) dO(T+1)
-          if (i + 1 < n_pairs) ok = issue_dv(T + 1, 1u);
         }
         if (!ok) break;
         tc_commit(bar_acc_full);
@@ -262,37 +225,33 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   } else {
     // ------------------------------------------------------- element-wise warps 0-7
     const int lg = warp & 3, ch = warp >> 2;
-    const int r = lg * 32 + lane;  // TMEM lane: key row for S^T/dP^T/dV/dK, query row for dQ
+    const int r = lg * 32 + lane;  // TMEM lane = key row
     const uint32_t lane_off = (uint32_t)(lg * 32) << 16;
-    const uint32_t stage_buf = sDs + warp * 4096;  // this warp's 32 x 128-byte dQ staging rows
-    uint8_t *stage_gen = smem_raw + SM::kOffDs + warp * 4096;
     uint32_t ic = 0, T = 0;
     bool ok = true;
     float pr[64];  // P^T of the current pair: key r, query columns 64*ch .. 64*ch+63
 
     // P^T(Tn) from S^T(Tn): wait, load, exponentiate, store bf16 over S^T, signal
     auto make_p = [&](uint32_t Tn, int q_base, int kv_pos0, int mode, bool key_valid) -> bool {
-      const uint32_t st = Tn % kBwdStages;
-      if (!mbar_wait(bar_q_full + 8 * st, (Tn / kBwdStages) & 1, ab, WAIT_BWD_QDO_FULL)) return false;  // row statistics landed
+      const uint32_t st = Tn % NST;
+      if (!mbar_wait(bar_q_full + 8 * st, (Tn / NST) & 1, ab, WAIT_BWD_QDO_FULL)) return false;  // row statistics landed
       if (!mbar_wait(bar_s_full, Tn & 1, ab, WAIT_BWD_S_FULL)) return false;
       tc_fence_after();
       const float *lse2 = reinterpret_cast<const float *>(smem_raw + SM::kOffStats + st * 1024) + ch * 64;
       // query column (inside the tile) from which this key is visible
       const int lo = mode ? 0 : (kv_pos0 + r - q_base);
       const bool all_visible = key_valid && lo <= ch * 64;
+      uint32_t sv[64];
+      tmem_ld32(tR0 + lane_off + ch * 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+      tmem_ld32(tR0 + lane_off + ch * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+      tc_wait_ld();
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t sv[32];
-        tmem_ld32(tR0 + lane_off + ch * 64 + c * 32, sv);
-        tc_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-          const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + c * 32 + i);
-          pr[c * 32 + i + 0] = ex2(__uint_as_float(sv[i + 0]) * p.scale_log2 - l4.x);
-          pr[c * 32 + i + 1] = ex2(__uint_as_float(sv[i + 1]) * p.scale_log2 - l4.y);
-          pr[c * 32 + i + 2] = ex2(__uint_as_float(sv[i + 2]) * p.scale_log2 - l4.z);
-          pr[c * 32 + i + 3] = ex2(__uint_as_float(sv[i + 3]) * p.scale_log2 - l4.w);
-        }
+      for (int i = 0; i < 64; i += 4) {
+        const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + i);
+        pr[i + 0] = ex2(fmaf(__uint_as_float(sv[i + 0]), p.scale_log2, -l4.x));
+        pr[i + 1] = ex2(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -l4.y));
+        pr[i + 2] = ex2(fmaf(__uint_as_float(sv[i + 2]), p.scale_log2, -l4.z));
+        pr[i + 3] = ex2(fmaf(__uint_as_float(sv[i + 3]), p.scale_log2, -l4.w));
       }
       if (!all_visible) {
 #pragma unroll
@@ -318,107 +277,59 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const bool key_valid = r < kv_rows;
       bool first = true;
       for (int sg = seg0; sg < seg0 + nseg && ok; ++sg) {
-        const int s_tok0 = p.segs[3 * sg], s_len = p.segs[3 * sg + 1];
+        const int s_len = p.segs[3 * sg + 1];
         const int nqt = (s_len + 127) >> 7;
         const int qt0 = mode ? 0 : (kv_pos0 >> 7);
         for (int qt = qt0; qt < nqt && ok; ++qt)
           for (int j = 0; j < rep; ++j, ++T) {
-            const uint32_t st = T % kBwdStages;
+            const uint32_t st = T % NST;
             if (first) {  // the item's first pair has no predecessor to pipeline behind
               ok = make_p(T, qt * 128, kv_pos0, mode, key_valid);
               if (!ok) break;
               first = false;
             }
-            // ---- dS^T(T) = P^T * (scale*dP^T - scale*delta): to shared memory (K-major rows of 64 queries)
+            // ---- dS^T(T) = P^T * (scale*dP^T - scale*delta), bf16 over dP^T in R1
             ok = mbar_wait(bar_dp_full, T & 1, ab, WAIT_BWD_S_FULL);
             if (!ok) break;
-            if (T > 0) {  // the dQ staging of pair T-1 shares the dS^T buffer
-              ok = mbar_wait(bar_stage_free, (T - 1) & 1, ab, WAIT_BWD_ROWS);
-              if (!ok) break;
-            }
             tc_fence_after();
             {
               const float *dl = reinterpret_cast<const float *>(smem_raw + SM::kOffStats + st * 1024) + 128 + ch * 64;
-              uint8_t *row = smem_raw + SM::kOffDs + ch * 16384 + r * 128;
+              uint32_t dpv[64];
+              tmem_ld32(tR1 + lane_off + ch * 64, *reinterpret_cast<uint32_t(*)[32]>(&dpv[0]));
+              tmem_ld32(tR1 + lane_off + ch * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&dpv[32]));
+              tc_wait_ld();
 #pragma unroll
               for (int c = 0; c < 2; ++c) {
-                uint32_t dpv[32];
-                tmem_ld32(tR1 + lane_off + ch * 64 + c * 32, dpv);
-                tc_wait_ld();
                 uint32_t dd[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 4) {
                   const float4 d4 = *reinterpret_cast<const float4 *>(dl + c * 32 + i);
-                  const float a0 = pr[c * 32 + i + 0] * fmaf(__uint_as_float(dpv[i + 0]), p.scale, -d4.x);
-                  const float a1 = pr[c * 32 + i + 1] * fmaf(__uint_as_float(dpv[i + 1]), p.scale, -d4.y);
-                  const float a2 = pr[c * 32 + i + 2] * fmaf(__uint_as_float(dpv[i + 2]), p.scale, -d4.z);
-                  const float a3 = pr[c * 32 + i + 3] * fmaf(__uint_as_float(dpv[i + 3]), p.scale, -d4.w);
+                  const float a0 = pr[c * 32 + i + 0] * fmaf(__uint_as_float(dpv[c * 32 + i + 0]), p.scale, -d4.x);
+                  const float a1 = pr[c * 32 + i + 1] * fmaf(__uint_as_float(dpv[c * 32 + i + 1]), p.scale, -d4.y);
+                  const float a2 = pr[c * 32 + i + 2] * fmaf(__uint_as_float(dpv[c * 32 + i + 2]), p.scale, -d4.z);
+                  const float a3 = pr[c * 32 + i + 3] * fmaf(__uint_as_float(dpv[c * 32 + i + 3]), p.scale, -d4.w);
                   dd[i / 2] = pack_bf16(a0, a1);
                   dd[i / 2 + 1] = pack_bf16(a2, a3);
                 }
-#pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                  const int chunk = c * 4 + v;
-                  *reinterpret_cast<uint4 *>(row + ((chunk ^ (r & 7)) << 4)) = make_uint4(dd[4 * v], dd[4 * v + 1], dd[4 * v + 2], dd[4 * v + 3]);
-                }
+                tmem_st16(tR1 + lane_off + ch * 64 + c * 16, dd);
               }
             }
-            fence_proxy_async_smem();
+            tc_wait_st();
             tc_fence_before();
             mbar_arrive(bar_ds_ready);
             // ---- P^T(T+1), if the item has another pair (same iteration order as the other roles)
             {
-              int nqt2 = qt, j2 = j + 1, sg2 = sg;
+              int qt2 = qt, j2 = j + 1;
               bool more = true;
-              if (j2 == rep) { j2 = 0; ++nqt2; }
-              int q_base2 = nqt2 * 128;
-              if (nqt2 >= nqt) {
-                ++sg2;
-                if (sg2 < seg0 + nseg) q_base2 = qt0 * 128; else more = false;
+              if (j2 == rep) { j2 = 0; ++qt2; }
+              int q_base2 = qt2 * 128;
+              if (qt2 >= nqt) {
+                if (sg + 1 < seg0 + nseg) q_base2 = qt0 * 128; else more = false;
               }
               if (more) {
                 ok = make_p(T + 1, q_base2, kv_pos0, mode, key_valid);
                 if (!ok) break;
               }
-            }
-            // ---- drain dQ(T): thread = query row r, columns 64*ch.. of d; fp32 reduce-add by TMA
-            ok = mbar_wait(bar_dq_full, T & 1, ab, WAIT_BWD_MMA2);
-            if (!ok) break;
-            tc_fence_after();
-            {
-              const int head = kvh * rep + j;
-              const int tok_row = s_tok0 + qt * 128 + lg * 32;
-              constexpr int ROUNDS = D / 64;  // each round: 32 columns per warp
-#pragma unroll
-              for (int rd = 0; rd < ROUNDS; ++rd) {
-                const int col0 = (ROUNDS == 2) ? ch * 64 + rd * 32 : ch * 32;
-                uint32_t v[32];
-                tmem_ld32(tR1 + lane_off + col0, v);
-                tc_wait_ld();
-                if (rd == ROUNDS - 1) {  // R1 fully read by this thread: dP(T+1) may overwrite it
-                  tc_fence_before();
-                  mbar_arrive(bar_drained);
-                }
-                if (rd > 0) {  // staging rows still being read by the previous round's reduce
-                  if (lane == 0) bulk_wait_read0();
-                  __syncwarp();
-                }
-                uint8_t *srow = stage_gen + lane * 128;
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                  *reinterpret_cast<uint4 *>(srow + ((q ^ (lane & 7)) << 4)) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                  tma_reduce_add_3d(&tm_dq, stage_buf, col0, head, tok_row);
-                  bulk_commit();
-                }
-              }
-              if (lane == 0) {
-                bulk_wait_read0();
-                mbar_arrive(bar_stage_free);
-              }
-              __syncwarp();
             }
           }
       }
@@ -463,7 +374,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       tc_fence_before();
       mbar_arrive(bar_acc_empty);
     }
-    if (lane == 0) bulk_wait0();  // all reduce-adds of this warp have been performed
   }
 
   __syncwarp();
@@ -502,7 +412,7 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16 *o, const __nv_bfloat1
   }
 }
 
-// fp32 -> bf16 (dQ accumulator, optional bf16 copies of the prompt gradients)
+// fp32 -> bf16 (optional bf16 copies of the prompt gradients)
 __global__ void cast_bf16_kernel(const float *src, __nv_bfloat16 *dst, long long n4) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n4) return;

@@ -11,8 +11,10 @@
 // Canonical item order (ids are positions in this order):
 //   prefill fwd : group, kv head, query tile, query head inside the kv head
 //   replay  fwd : group, kv head, branch, query tile, query head, prompt-KV shard
-//   replay  bwd : group, kv head, [prompt kv tiles, then branch by branch its kv tiles]
-//   prefill bwd : group, kv head, kv tile
+//   replay  bwd : group, kv head, [prompt kv tiles, then branch by branch its kv tiles]   (dK, dV)
+//   prefill bwd : group, kv head, kv tile                                                 (dK, dV)
+//   replay  dQ  : group, kv head, branch, query tile, query head   (never sharded)
+//   prefill dQ  : as prefill fwd
 // Assignment: ids sorted by (weight descending, id ascending); each goes to the
 // lane with the smallest load so far (lowest lane index on ties).  Inside a
 // lane items run in ascending id, which keeps lanes on the same kv head at
@@ -128,9 +130,10 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
 
   Sched &pf = p->sched[SCHED_PREFILL_FWD], &rf = p->sched[SCHED_REPLAY_FWD];
   Sched &rb = p->sched[SCHED_REPLAY_BWD], &pb = p->sched[SCHED_PREFILL_BWD];
-  pf.item_ints = rf.item_ints = AUGTREE_FWD_ITEM_INTS;
+  Sched &rq = p->sched[SCHED_REPLAY_DQ], &pq = p->sched[SCHED_PREFILL_DQ];
+  pf.item_ints = rf.item_ints = rq.item_ints = pq.item_ints = AUGTREE_FWD_ITEM_INTS;
   rb.item_ints = pb.item_ints = AUGTREE_BWD_ITEM_INTS;
-  pf.items.clear(); rf.items.clear(); rb.items.clear(); pb.items.clear();
+  pf.items.clear(); rf.items.clear(); rb.items.clear(); pb.items.clear(); rq.items.clear(); pq.items.clear();
 
   for (int g = 0; g < ng; ++g) {
     const int P = p->prompt_len[g], p0 = p->cu_p[g];
@@ -144,6 +147,11 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
           const int32_t it[AUGTREE_FWD_ITEM_INTS] = {p0 + t * kTileQ, t * kTileQ, rows, c * rep + j, 0, 0, p0, blen,
                                                      0, 1, cdiv(blen, kTileKV), c};
           pf.items.insert(pf.items.end(), it, it + AUGTREE_FWD_ITEM_INTS);
+          // dQ item: the same unit; field 8 is the tile's index in the per-tile row statistics
+          int32_t dq[AUGTREE_FWD_ITEM_INTS];
+          std::copy(it, it + AUGTREE_FWD_ITEM_INTS, dq);
+          dq[8] = p->seg_prefill[3 * g + 2] + t;
+          pq.items.insert(pq.items.end(), dq, dq + AUGTREE_FWD_ITEM_INTS);
         }
       }
       // ---- replay forward ----
@@ -153,6 +161,11 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
         for (int t = 0; t < cdiv(R, kTileQ); ++t) {
           const int rows = std::min(kTileQ, R - t * kTileQ);
           const int blen = t * kTileQ + rows;
+          for (int j = 0; j < rep; ++j) {  // dQ item: never sharded, field 8 = statistics tile index
+            const int32_t dq[AUGTREE_FWD_ITEM_INTS] = {r0 + t * kTileQ, t * kTileQ, rows, c * rep + j, p0, P, r0, blen,
+                                                       p->seg_replay[3 * b + 2] + t, 1, cdiv(P, kTileKV) + cdiv(blen, kTileKV), c};
+            rq.items.insert(rq.items.end(), dq, dq + AUGTREE_FWD_ITEM_INTS);
+          }
           for (int j = 0; j < rep; ++j)
             for (int s = 0; s < ns; ++s) {
               const int a0 = s * shard_tiles[g] * kTileKV;
@@ -197,6 +210,8 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
     assign_lanes(rf, 10, p->n_lanes);
     assign_lanes(rb, 7, p->n_lanes);
     assign_lanes(pb, 7, p->n_lanes);
+    assign_lanes(rq, 10, p->n_lanes);
+    assign_lanes(pq, 10, p->n_lanes);
   }
 
   // scratch sizes (bytes, each region 256-byte aligned)
@@ -206,9 +221,10 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
   if (p->max_splits > 1)
     p->ws_fwd = al((size_t)p->max_splits * (size_t)tr * hq * dd * 4) + al((size_t)p->max_splits * (size_t)tr * hq * 4);
   const size_t tmax = (size_t)std::max<int64_t>(tp, tr);
-  // backward: dq accumulator fp32 [tokens,H_q,d]; row statistics [H_q][tiles][2][128] fp32
+  // backward: row statistics [H_q][tiles][2][128] fp32
   const size_t ntile = std::max(p->tiles_replay.size(), p->tiles_prefill.size()) / 2;
-  p->ws_bwd = al(tmax * hq * dd * 4) + al(hq * ntile * 2 * kTileQ * 4);
+  p->ws_bwd = al(hq * ntile * 2 * kTileQ * 4);
+  (void)tmax; (void)dd;
   return AUGTREE_OK;
 }
 

@@ -10,7 +10,8 @@ namespace augtree {
 constexpr int kTileQ = 128;   // query rows per tile
 constexpr int kTileKV = 128;  // keys per tile
 
-enum { SCHED_PREFILL_FWD = 0, SCHED_REPLAY_FWD = 1, SCHED_REPLAY_BWD = 2, SCHED_PREFILL_BWD = 3, SCHED_COUNT = 4 };
+enum { SCHED_PREFILL_FWD = 0, SCHED_REPLAY_FWD = 1, SCHED_REPLAY_BWD = 2, SCHED_PREFILL_BWD = 3, SCHED_REPLAY_DQ = 4, SCHED_PREFILL_DQ = 5,
+       SCHED_COUNT = 6 };
 
 struct Sched {
   int item_ints = 0;
@@ -26,7 +27,7 @@ struct Sched {
 struct Timing {
   bool on = false;
   std::vector<void *> ev[SCHED_COUNT];  // cudaEvent_t start/stop pairs, in launch order
-  size_t used[SCHED_COUNT] = {0, 0, 0, 0};
+  size_t used[SCHED_COUNT] = {};
 };
 
 }  // namespace augtree

@@ -135,6 +135,34 @@ __device__ __forceinline__ uint64_t make_sdesc(uint32_t saddr, uint32_t lbo_byte
          (1ull << 46) | (2ull << 61);
 }
 
+// The same descriptor as two 32-bit words, so that the issuing thread only adds
+// a constant per K step: the high word depends on the layout alone, the low
+// word is address | LBO.
+__host__ __device__ constexpr uint32_t sdesc_hi(uint32_t sbo_bytes) { return (sbo_bytes >> 4) | (1u << 14) | (2u << 29); }
+__device__ __forceinline__ uint32_t sdesc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+constexpr uint32_t kDescHi = sdesc_hi(1024);  // every operand tile here: 1024 bytes between 8-row groups
+// low-word increments (bytes >> 4) of the K steps: K-major tiles advance 32 bytes inside a 64-element
+// box and 16 KB to the next box; MN-major tiles advance 16 rows of 128 bytes
+__host__ __device__ constexpr uint32_t kstep_kmajor(int k) { return (uint32_t)(((k >> 2) * 16384 + (k & 3) * 32) >> 4); }
+__host__ __device__ constexpr uint32_t kstep_mnmajor(int k) { return (uint32_t)((k * 2048) >> 4); }
+
+__device__ __forceinline__ void mma_ss2(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(acc), "r"(kDescHi) : "memory");
+}
+__device__ __forceinline__ void mma_ts2(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "mov.b64 db, {%2, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(acc), "r"(kDescHi) : "memory");
+}
+
 // TMEM <-> registers, 32 lanes x 32 columns of 32 bits: thread t of the warp
 // gets lane (32 * (warp % 4) + t), columns [col, col + 32).
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {

@@ -75,7 +75,8 @@ def test_tables_bit_exact(binding, pl, bl, hq, hkv, lanes, splits):
     assert (plan.metadata(B.TBL_REPLAY_SEGMENTS).reshape(-1, 3) == ref["seg_replay"]).all()
     assert (plan.metadata(B.TBL_PREFILL_SEGMENTS).reshape(-1, 3) == ref["seg_prefill"]).all()
     for base, key, w, wf in [(B.TBL_PREFILL_FWD_ITEMS, "prefill_fwd", 12, 10), (B.TBL_REPLAY_FWD_ITEMS, "replay_fwd", 12, 10),
-                             (B.TBL_REPLAY_BWD_ITEMS, "replay_bwd", 8, 7), (B.TBL_PREFILL_BWD_ITEMS, "prefill_bwd", 8, 7)]:
+                             (B.TBL_REPLAY_BWD_ITEMS, "replay_bwd", 8, 7), (B.TBL_PREFILL_BWD_ITEMS, "prefill_bwd", 8, 7),
+                             (B.TBL_REPLAY_DQ_ITEMS, "replay_dq", 12, 10), (B.TBL_PREFILL_DQ_ITEMS, "prefill_dq", 12, 10)]:
         items = plan.metadata(base).reshape(-1, w)
         assert items.shape == ref[key].shape and (items == ref[key]).all(), key
         ptr, order = packing.assign_lanes(ref[key][:, wf], lanes)
@@ -102,6 +103,7 @@ def test_item_weights_count_visible_pairs():
         return tot
     assert fwd_pairs(ref["prefill_fwd"]) == pre * hq
     assert fwd_pairs(ref["replay_fwd"]) == rep * hq
+    assert fwd_pairs(ref["replay_dq"]) == rep * hq and fwd_pairs(ref["prefill_dq"]) == pre * hq
 
     def bwd_pairs(items, segs):
         tot = 0
