@@ -3,9 +3,10 @@
 Written from the rules, not from the library's source: the tests demand that
 the library's tables equal these bit for bit.
 
-Rules.  Tiles are 128 query rows by 128 keys.  A forward item is one (query
-tile, query head[, prompt-KV shard]); its weight is the number of KV tiles it
-visits.  A backward item is one (KV tile, KV head); its weight is the number of
+Rules.  Tiles are 128 query rows by 128 keys.  A forward item is one (pair of
+consecutive query tiles, query head[, prompt-KV shard]); its weight is the
+number of (query tile, KV tile) visits.  A dQ item is one (query tile, query
+head), weighted by its KV tiles.  A backward item is one (KV tile, KV head); its weight is the number of
 (query tile, query head) visits.  Items are listed in a canonical order, then
 assigned to lanes largest weight first (ties: lower id first), each to the lane
 with the least load so far (ties: lowest lane), following the balanced
@@ -19,6 +20,7 @@ import heapq
 import numpy as np
 
 TQ = TK = 128
+TQF = 256   # forward units cover two query tiles
 
 
 def _cdiv(a, b):
@@ -49,11 +51,15 @@ def build_tables(prompt_len, branch_len, h_q, h_kv, kv_splits=1):
         ns = _cdiv(na, shard_tiles)
         gsplits.append(ns)
         for c in range(h_kv):
-            for t in range(_cdiv(P, TQ)):
+            for t in range(_cdiv(P, TQF)):      # forward units: two query tiles
+                rows = min(TQF, P - t * TQF)
+                vis = t * TQF + rows
+                for j in range(rep):
+                    pf.append([p0 + t * TQF, t * TQF, rows, c * rep + j, 0, 0, p0, vis, 0, 1, _cdiv(vis, TK) * _cdiv(rows, TQ), c])
+            for t in range(_cdiv(P, TQ)):       # dQ units: one query tile
                 rows = min(TQ, P - t * TQ)
                 vis = t * TQ + rows
                 for j in range(rep):
-                    pf.append([p0 + t * TQ, t * TQ, rows, c * rep + j, 0, 0, p0, vis, 0, 1, _cdiv(vis, TK), c])
                     pq.append([p0 + t * TQ, t * TQ, rows, c * rep + j, 0, 0, p0, vis, ptile0[g] + t, 1, _cdiv(vis, TK), c])
             for bi in range(cu_b[g], cu_b[g + 1]):
                 R, r0 = flat[bi], cu_r[bi]
@@ -63,13 +69,16 @@ def build_tables(prompt_len, branch_len, h_q, h_kv, kv_splits=1):
                     for j in range(rep):
                         rq.append([r0 + t * TQ, t * TQ, rows, c * rep + j, p0, P, r0, vis, rtile0[bi] + t, 1,
                                    _cdiv(P, TK) + _cdiv(vis, TK), c])
+                for t in range(_cdiv(R, TQF)):
+                    rows = min(TQF, R - t * TQF)
+                    vis = t * TQF + rows
                     for j in range(rep):
                         for s in range(ns):
                             a0 = s * shard_tiles * TK
                             alen = min(P - a0, shard_tiles * TK)
                             bl = vis if s == ns - 1 else 0
-                            rf.append([r0 + t * TQ, t * TQ, rows, c * rep + j, p0 + a0, alen, r0, bl, s, ns,
-                                       _cdiv(alen, TK) + _cdiv(bl, TK), c])
+                            rf.append([r0 + t * TQF, t * TQF, rows, c * rep + j, p0 + a0, alen, r0, bl, s, ns,
+                                       (_cdiv(alen, TK) + _cdiv(bl, TK)) * _cdiv(rows, TQ), c])
             b0, b1 = cu_b[g], cu_b[g + 1]
             if b1 > b0:
                 visits = sum(_cdiv(flat[bi], TQ) * rep for bi in range(b0, b1))

@@ -139,40 +139,49 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
     const int P = p->prompt_len[g], p0 = p->cu_p[g];
     const int nqt_p = cdiv(P, kTileQ);
     for (int c = 0; c < p->h_kv; ++c) {
-      // ---- prefill forward ----
+      // ---- prefill forward: units of two query tiles (256 rows) ----
+      for (int t = 0; t < cdiv(P, kTileQF); ++t) {
+        const int rows = std::min(kTileQF, P - t * kTileQF);
+        const int blen = t * kTileQF + rows;
+        for (int j = 0; j < rep; ++j) {
+          const int32_t it[AUGTREE_FWD_ITEM_INTS] = {p0 + t * kTileQF, t * kTileQF, rows, c * rep + j, 0, 0, p0, blen,
+                                                     0, 1, cdiv(blen, kTileKV) * cdiv(rows, kTileQ), c};
+          pf.items.insert(pf.items.end(), it, it + AUGTREE_FWD_ITEM_INTS);
+        }
+      }
+      // ---- prefill dQ: units of one query tile; field 8 is the tile's index in the per-tile row statistics ----
       for (int t = 0; t < nqt_p; ++t) {
         const int rows = std::min(kTileQ, P - t * kTileQ);
         const int blen = t * kTileQ + rows;
         for (int j = 0; j < rep; ++j) {
-          const int32_t it[AUGTREE_FWD_ITEM_INTS] = {p0 + t * kTileQ, t * kTileQ, rows, c * rep + j, 0, 0, p0, blen,
-                                                     0, 1, cdiv(blen, kTileKV), c};
-          pf.items.insert(pf.items.end(), it, it + AUGTREE_FWD_ITEM_INTS);
-          // dQ item: the same unit; field 8 is the tile's index in the per-tile row statistics
-          int32_t dq[AUGTREE_FWD_ITEM_INTS];
-          std::copy(it, it + AUGTREE_FWD_ITEM_INTS, dq);
-          dq[8] = p->seg_prefill[3 * g + 2] + t;
+          const int32_t dq[AUGTREE_FWD_ITEM_INTS] = {p0 + t * kTileQ, t * kTileQ, rows, c * rep + j, 0, 0, p0, blen,
+                                                     p->seg_prefill[3 * g + 2] + t, 1, cdiv(blen, kTileKV), c};
           pq.items.insert(pq.items.end(), dq, dq + AUGTREE_FWD_ITEM_INTS);
         }
       }
-      // ---- replay forward ----
+      // ---- replay forward (256-row units, optionally sharded over the prompt KV) and replay dQ (128-row units) ----
       for (int b = p->cu_b[g]; b < p->cu_b[g + 1]; ++b) {
         const int R = p->branch_len[b], r0 = p->cu_r[b];
         const int ns = p->group_splits[g];
         for (int t = 0; t < cdiv(R, kTileQ); ++t) {
           const int rows = std::min(kTileQ, R - t * kTileQ);
           const int blen = t * kTileQ + rows;
-          for (int j = 0; j < rep; ++j) {  // dQ item: never sharded, field 8 = statistics tile index
+          for (int j = 0; j < rep; ++j) {
             const int32_t dq[AUGTREE_FWD_ITEM_INTS] = {r0 + t * kTileQ, t * kTileQ, rows, c * rep + j, p0, P, r0, blen,
                                                        p->seg_replay[3 * b + 2] + t, 1, cdiv(P, kTileKV) + cdiv(blen, kTileKV), c};
             rq.items.insert(rq.items.end(), dq, dq + AUGTREE_FWD_ITEM_INTS);
           }
+        }
+        for (int t = 0; t < cdiv(R, kTileQF); ++t) {
+          const int rows = std::min(kTileQF, R - t * kTileQF);
+          const int blen = t * kTileQF + rows;
           for (int j = 0; j < rep; ++j)
             for (int s = 0; s < ns; ++s) {
               const int a0 = s * shard_tiles[g] * kTileKV;
               const int alen = std::min(P - a0, shard_tiles[g] * kTileKV);
               const int bl = (s == ns - 1) ? blen : 0;
-              const int32_t it[AUGTREE_FWD_ITEM_INTS] = {r0 + t * kTileQ, t * kTileQ, rows, c * rep + j, p0 + a0, alen,
-                                                         r0, bl, s, ns, cdiv(alen, kTileKV) + cdiv(bl, kTileKV), c};
+              const int32_t it[AUGTREE_FWD_ITEM_INTS] = {r0 + t * kTileQF, t * kTileQF, rows, c * rep + j, p0 + a0, alen,
+                                                         r0, bl, s, ns, (cdiv(alen, kTileKV) + cdiv(bl, kTileKV)) * cdiv(rows, kTileQ), c};
               rf.items.insert(rf.items.end(), it, it + AUGTREE_FWD_ITEM_INTS);
             }
         }

@@ -8,6 +8,7 @@
 namespace augtree {
 
 constexpr int kTileQ = 128;   // query rows per tile
+constexpr int kTileQF = 256;  // query rows per forward unit (two tiles share every K/V tile they load)
 constexpr int kTileKV = 128;  // keys per tile
 
 enum { SCHED_PREFILL_FWD = 0, SCHED_REPLAY_FWD = 1, SCHED_REPLAY_BWD = 2, SCHED_PREFILL_BWD = 3, SCHED_REPLAY_DQ = 4, SCHED_PREFILL_DQ = 5,
