@@ -163,6 +163,25 @@ def run_reference(args, w):
 
 
 # --------------------------------------------------------------------------- #
+def rank_workload(w, rank):
+    """Rank r replays its own trees of the same shape: same lengths, seed + r (weak scaling, no exchange)."""
+    return wl.Workload(w.name, w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, w.seed + rank, w.note, dict(w.extra))
+
+
+def max_over_ranks(ms, dist, device="cuda"):
+    """The job's time is the slowest rank's."""
+    if dist is None:
+        return float(ms)
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tflops(flops_per_rank, world, ms_per_step):
+    """Whole-job useful TFLOP/s: every rank does flops_per_rank in ms_per_step (the max over ranks)."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
 def time_steps(step_fn, steps, warmup, dist, sampler_index=None):
     """W warm-up steps, then K steps between two events, bracketed by barrier + synchronize; max over ranks."""
     for _ in range(warmup):
@@ -186,11 +205,7 @@ def time_steps(step_fn, steps, warmup, dist, sampler_index=None):
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), dist)
     return ms, (sampler.summary() if sampler else None)
 
 
@@ -227,7 +242,7 @@ def main():
         import torch.distributed as dist_mod
         dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
         dist = dist_mod
-    w.seed += rank  # every rank replays its own trees of the same shape
+    w = rank_workload(w, rank)
     fl = useful_flops(w)
     pk = peaks()
 
@@ -253,7 +268,7 @@ def main():
     kt = [plan.kernel_time(k) for k in range(6)]
     plan.set_timing(False)
     ms_step = ms / args.steps
-    value = world * fl["total"] / (ms_step * 1e-3) / 1e12
+    value = aggregate_tflops(fl["total"], world, ms_step)
 
     # dominant kernel: the replay backward tile kernel
     names = ["prefill_fwd", "replay_fwd", "replay_bwd_dkdv", "prefill_bwd_dkdv", "replay_bwd_dq", "prefill_bwd_dq"]
@@ -286,7 +301,7 @@ def main():
     if not args.no_e2e:
         ms_e2e, _ = time_steps(step_e2e, max(3, args.steps // 2), 3, dist)
         ms_e2e /= max(3, args.steps // 2)
-        e2e = {"value": world * fl["total"] / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+        e2e = {"value": aggregate_tflops(fl["total"], world, ms_e2e), "unit": "TFLOP/s", "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     # ---- flattened no-reuse baseline: same kernels, prompt duplicated per branch

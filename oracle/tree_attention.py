@@ -248,6 +248,43 @@ def dq_row(tb, q_p, k_p, v_p, do_p, q_r, k_r, v_r, do_r, kind, token, head):
     return tb.scale * (ds @ k)
 
 
+def dkv_key(tb, q_p, k_p, v_p, do_p, q_r, k_r, v_r, do_r, kind, token, kv_head):
+    """dK and dV of one key (kind 'p' prompt / 'r' response, packed token index, KV head).
+
+    Sums, over every query row that sees the key and every query head of the KV
+    head, p_ab * dO_a (dV) and scale * dS_ab * q_a (dK), each row's softmax taken
+    over that row's full visible key set.  For a prompt key the rows are the later
+    prompt rows and every response row of every branch of the group (Eq. 2).
+    Cost grows with the number of rows, so use it for keys few rows can see.
+    """
+    hq, hkv = tb.h_q, tb.h_kv
+    rep = hq // hkv
+    d = tb.head_dim
+    dk, dv = np.zeros(d), np.zeros(d)
+    if kind == "p":
+        g = int(np.searchsorted(tb.cu_p, token, side="right") - 1)
+        rows = [("p", a) for a in range(token, int(tb.cu_p[g + 1]))]
+        for b in range(int(tb.cu_b[g]), int(tb.cu_b[g + 1])):
+            rows += [("r", a) for a in range(int(tb.cu_r[b]), int(tb.cu_r[b + 1]))]
+        kvec = np.asarray(k_p[token, kv_head], dtype=np.float64)
+        vvec = np.asarray(v_p[token, kv_head], dtype=np.float64)
+    else:
+        b = int(np.searchsorted(tb.cu_r, token, side="right") - 1)
+        rows = [("r", a) for a in range(token, int(tb.cu_r[b + 1]))]
+        kvec = np.asarray(k_r[token, kv_head], dtype=np.float64)
+        vvec = np.asarray(v_r[token, kv_head], dtype=np.float64)
+    for (rk, a) in rows:
+        for h in range(kv_head * rep, (kv_head + 1) * rep):
+            o, lse = forward_row(tb, q_p, k_p, v_p, q_r, k_r, v_r, rk, a, h)
+            q = np.asarray((q_p if rk == "p" else q_r)[a, h], dtype=np.float64)
+            do = np.asarray((do_p if rk == "p" else do_r)[a, h], dtype=np.float64)
+            p_ab = np.exp(tb.scale * (q @ kvec) - lse)
+            dv += p_ab * do
+            ds = p_ab * (do @ vvec - do @ o)
+            dk += tb.scale * ds * q
+    return dk, dv
+
+
 # --------------------------------------------------------------------------- #
 # Second and third formulations, used only to pin the one above.
 # --------------------------------------------------------------------------- #

@@ -1,0 +1,62 @@
+"""The N > 1 path of the benchmark on CPU: two gloo ranks (no GPU, no data-path collective).
+
+Ranks replay independent groups, so the only cross-rank steps are the barrier and the max over ranks of
+the timed region; this checks the sharding rule and that reduction with world_size 2 over 127.0.0.1.
+"""
+import os
+import socket
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import bench
+from paper_2609_33133_b200 import workloads as wl
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    w = bench.rank_workload(wl.config(1), rank)
+    local_ms = 10.0 + 5.0 * rank                      # rank 1 is the slow one
+    ms = bench.max_over_ranks(local_ms, dist, device="cpu")
+    val = bench.aggregate_tflops(bench.useful_flops(w)["total"], world, ms)
+    out.put((rank, w.seed, w.prompt_len, ms, val))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_shard_and_reduce():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    base = wl.config(1)
+    assert [r[1] for r in res] == [base.seed, base.seed + 1]          # own trees per rank ...
+    assert all(r[2] == base.prompt_len for r in res)                  # ... of the same shape (weak scaling)
+    assert all(abs(r[3] - 15.0) < 1e-9 for r in res)                  # max over ranks
+    fl = bench.useful_flops(base)["total"]
+    assert all(abs(r[4] - 2 * fl / 15e-3 / 1e12) < 1e-9 for r in res)  # whole-job value over the slowest rank's time
+
+
+def test_flop_accounting_matches_oracle_pair_count():
+    from oracle import tree_attention as ora
+    for i in (1, 2, 3):
+        w = wl.config(i)
+        pre, rep, flat = ora.valid_pairs(ora.TreeBatch(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim))
+        fl = bench.useful_flops(w)
+        assert fl["total"] == 14 * w.head_dim * w.h_q * (pre + rep)
+        assert abs(fl["reuse_factor"] - flat / (pre + rep)) < 1e-12
+    assert abs(bench.useful_flops(wl.config(2))["total"] / 1e12 - 9.2606) < 1e-3

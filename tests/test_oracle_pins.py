@@ -209,6 +209,16 @@ def test_row_forms_match_matrix_form():
         np.testing.assert_allclose(dq, res["dq" + sfx][tok, h], rtol=1e-10, atol=1e-11)
 
 
+def test_key_form_matches_matrix_form():
+    tb, t = _rand_tree(11, [6, 4], [[3, 5], [2]], 4, 2, 8)
+    res = _run(tb, t)
+    for kind, tok, c in [("p", 0, 0), ("p", 5, 1), ("p", 8, 0), ("r", 0, 1), ("r", 7, 0), ("r", 9, 1)]:
+        dk, dv = ora.dkv_key(tb, t["q_p"], t["k_p"], t["v_p"], t["do_p"], t["q_r"], t["k_r"], t["v_r"], t["do_r"], kind, tok, c)
+        sfx = "_p" if kind == "p" else "_r"
+        np.testing.assert_allclose(dk, res["dk" + sfx][tok, c], rtol=1e-10, atol=1e-11)
+        np.testing.assert_allclose(dv, res["dv" + sfx][tok, c], rtol=1e-10, atol=1e-11)
+
+
 # --- work accounting: flattening repeats the prompt pairs G times (Sec. 1) ---
 def test_redundancy_fraction():
     for G, want in [(8, 0.875), (64, 0.984375)]:
