@@ -95,8 +95,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       mbar_init(bar_q_full + 8 * s, 1); mbar_init(bar_q_empty + 8 * s, 1);
       mbar_init(bar_do_full + 8 * s, 1); mbar_init(bar_do_empty + 8 * s, 1);
     }
-    mbar_init(bar_s_full, 1); mbar_init(bar_p_ready, 256); mbar_init(bar_dp_full, 1); mbar_init(bar_ds_ready, 256);
-    mbar_init(bar_acc_full, 1); mbar_init(bar_acc_empty, 256);
+    mbar_init(bar_s_full, 1); mbar_init(bar_p_ready, 8); mbar_init(bar_dp_full, 1); mbar_init(bar_ds_ready, 8);
+    mbar_init(bar_acc_full, 1); mbar_init(bar_acc_empty, 8);
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -267,7 +267,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       }
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_p_ready);
+      warp_arrive(bar_p_ready);
       return true;
     };
 
@@ -316,7 +316,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             }
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(bar_ds_ready);
+            warp_arrive(bar_ds_ready);
             // ---- P^T(T+1), if the item has another pair (same iteration order as the other roles)
             {
               int qt2 = qt, j2 = j + 1;
@@ -372,7 +372,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
       }
       tc_fence_before();
-      mbar_arrive(bar_acc_empty);
+      warp_arrive(bar_acc_empty);
     }
   }
 

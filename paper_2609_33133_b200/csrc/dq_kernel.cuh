@@ -80,11 +80,11 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    mbar_init(bar_qdo_full, 1); mbar_init(bar_qdo_empty, 256); mbar_init(bar_qt_ready, 256);
+    mbar_init(bar_qdo_full, 1); mbar_init(bar_qdo_empty, 8); mbar_init(bar_qt_ready, 8);
     for (int s = 0; s < NK; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 1); }
     for (int s = 0; s < NV; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 1); }
-    mbar_init(bar_s_full, 1); mbar_init(bar_s_read, 256); mbar_init(bar_dp_full, 1); mbar_init(bar_ds_ready, 256);
-    mbar_init(bar_dq_full, 1); mbar_init(bar_dq_empty, 256);
+    mbar_init(bar_s_full, 1); mbar_init(bar_s_read, 8); mbar_init(bar_dp_full, 1); mbar_init(bar_ds_ready, 8);
+    mbar_init(bar_dq_full, 1); mbar_init(bar_dq_empty, 8);
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -228,8 +228,8 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       }
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_qt_ready);
-      mbar_arrive(bar_qdo_empty);
+      warp_arrive(bar_qt_ready);
+      warp_arrive(bar_qdo_empty);
       for (int i = 0; i < n; ++i, ++T) {
         // ---- P(T): registers only
         ok = mbar_wait(bar_s_full, T & 1, ab, WAIT_DQ_S);
@@ -242,7 +242,7 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           tmem_ld32(tS + lane_off + ch * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
           tc_wait_ld();
           tc_fence_before();
-          mbar_arrive(bar_s_read);
+          warp_arrive(bar_s_read);
           // number of leading key columns of this tile that the row sees
           const int limit = (i < nA) ? (a_len - i * 128) : (q_pos0 + r + 1 - (i - nA) * 128);
           const int lim = limit - ch * 64;
@@ -277,7 +277,7 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         }
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(bar_ds_ready);
+        warp_arrive(bar_ds_ready);
       }
       if (!ok) break;
       // ---- epilogue: dQ row r, columns (D/2)*ch .., rounded to bf16 once
@@ -304,7 +304,7 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         }
       }
       tc_fence_before();
-      mbar_arrive(bar_dq_empty);
+      warp_arrive(bar_dq_empty);
     }
   }
 

@@ -74,8 +74,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     mbar_init(bar_q_full, 1); mbar_init(bar_q_empty, 1);
     for (int s = 0; s < NS; ++s) { mbar_init(bar_kv_full + 8 * s, 1); mbar_init(bar_kv_empty + 8 * s, 1); }
     for (int g = 0; g < 2; ++g) {
-      mbar_init(bar_s_full + 8 * g, 1); mbar_init(bar_p_full + 8 * g, 128);
-      mbar_init(bar_o_full + 8 * g, 1); mbar_init(bar_o_empty + 8 * g, 128);
+      mbar_init(bar_s_full + 8 * g, 1); mbar_init(bar_p_full + 8 * g, 4);
+      mbar_init(bar_o_full + 8 * g, 1); mbar_init(bar_o_empty + 8 * g, 4);
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -291,7 +291,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         l += sum;
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(bar_p_full + 8 * g);
+        warp_arrive(bar_p_full + 8 * g);
       }
       if (!ok) break;
       // ---- epilogue: O / l, LSE = ln2 * (m + log2 l)
@@ -333,7 +333,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         else p.part_lse[((long long)split * p.h_q + head) * p.n_tok + tok] = lse;
       }
       tc_fence_before();
-      mbar_arrive(bar_o_empty + 8 * g);
+      warp_arrive(bar_o_empty + 8 * g);
     }
   }
 
