@@ -158,14 +158,12 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       uint32_t ic = 0, T = 0;
       bool ok = true;
       const uint32_t kk_lo = sdesc_lo(sK, 16), vk_lo = sdesc_lo(sV, 16);
-      auto issue_s = [&](uint32_t Tn) -> bool {  // S^T(Tn) = K Q^T -> R0
-        const uint32_t st = Tn % NST;
-        if (!mbar_wait(bar_q_full + 8 * st, (Tn / NST) & 1, ab, WAIT_BWD_QDO_FULL)) return false;
+      // Each group looks at the barrier of the group after it before its own last two MMAs (`have`), so
+      // that a hand-off which has already happened costs the tensor pipe nothing; only a look that fails
+      // turns into a wait between the groups.
+      auto need = [&](bool have, uint32_t bar, uint32_t par, int site) -> bool {
+        if (!have && !mbar_wait(bar, par, ab, site)) return false;
         tc_fence_after();
-        const uint32_t qk_lo = sdesc_lo(sQ0 + st * TILE, 16);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) mma_ss2(tR0, kk_lo + kstep_kmajor(k), qk_lo + kstep_kmajor(k), IDESC_ST, k > 0);
-        tc_commit(bar_s_full);
         return true;
       };
       for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
@@ -178,43 +176,69 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
         ok = mbar_wait(bar_kv_full, ic & 1, ab, WAIT_BWD_KV_FULL);
         if (!ok) break;
-        ok = issue_s(T);  // prologue: S^T of the item's first pair
-        for (int i = 0; i < n_pairs && ok; ++i, ++T) {
-          const uint32_t st = T % NST;
-          const uint32_t dok_lo = sdesc_lo(sDo0 + st * TILE, 16), dom_lo = sdesc_lo(sDo0 + st * TILE, 16384);
-          const uint32_t qm_lo = sdesc_lo(sQ0 + st * TILE, 16384);
-          const uint32_t acc0 = i > 0 ? 1u : 0u;
-          // ---- dP^T(T) = V dO^T -> R1
-          ok = mbar_wait(bar_do_full + 8 * st, (T / NST) & 1, ab, WAIT_BWD_QDO_FULL);
+        bool have_do = false;
+        {  // prologue: S^T of the item's first pair -> R0
+          const uint32_t st = T % NST, par = (T / NST) & 1;
+          ok = need(false, bar_q_full + 8 * st, par, WAIT_BWD_QDO_FULL);
           if (!ok) break;
-          tc_fence_after();
+          const uint32_t qk_lo = sdesc_lo(sQ0 + st * TILE, 16);
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) mma_ss2(tR1, vk_lo + kstep_kmajor(k), dok_lo + kstep_kmajor(k), IDESC_ST, k > 0);
+          for (int k = 0; k < D / 16; ++k) {
+            if (k == D / 16 - 2) have_do = mbar_test(bar_do_full + 8 * st, par);
+            mma_ss2(tR0, kk_lo + kstep_kmajor(k), qk_lo + kstep_kmajor(k), IDESC_ST, k > 0);
+          }
+          tc_commit(bar_s_full);
+        }
+        for (int i = 0; i < n_pairs && ok; ++i, ++T) {
+          const uint32_t st = T % NST, par = (T / NST) & 1;
+          const uint32_t st1 = (T + 1) % NST, par1 = ((T + 1) / NST) & 1;
+          const bool more = i + 1 < n_pairs;
+          const uint32_t dok_lo = sdesc_lo(sDo0 + st * TILE, 16), dom_lo = sdesc_lo(sDo0 + st * TILE, 16384);
+          const uint32_t qm_lo = sdesc_lo(sQ0 + st * TILE, 16384), qk1_lo = sdesc_lo(sQ0 + st1 * TILE, 16);
+          const uint32_t acc0 = i > 0 ? 1u : 0u;
+          bool have_p = false, have_q = false, have_ds = false;
+          // ---- dP^T(T) = V dO^T -> R1
+          ok = need(have_do, bar_do_full + 8 * st, par, WAIT_BWD_QDO_FULL);
+          if (!ok) break;
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {
+            if (k == D / 16 - 2) have_p = mbar_test(bar_p_ready, T & 1);
+            mma_ss2(tR1, vk_lo + kstep_kmajor(k), dok_lo + kstep_kmajor(k), IDESC_ST, k > 0);
+          }
           tc_commit(bar_dp_full);
           // ---- dV += P^T(T) dO(T)
-          ok = mbar_wait(bar_p_ready, T & 1, ab, WAIT_BWD_PDS_FULL);
-          if (!ok) break;
           if (i == 0 && ic > 0) {  // the previous item's dV/dK must have left TMEM
             ok = mbar_wait(bar_acc_empty, (ic - 1) & 1, ab, WAIT_BWD_ACC_EMPTY);
             if (!ok) break;
           }
-          tc_fence_after();
+          ok = need(have_p, bar_p_ready, T & 1, WAIT_BWD_PDS_FULL);
+          if (!ok) break;
 #pragma unroll
-          for (int k = 0; k < 8; ++k)  // query columns 16k..16k+15: P^T sits at R0 columns 8k (k<4) or 64+8(k-4)
+          for (int k = 0; k < 8; ++k) {  // query columns 16k..16k+15: P^T sits at R0 columns 8k (k<4) or 64+8(k-4)
+            if (k == 6) have_q = more && mbar_test(bar_q_full + 8 * st1, par1);
             mma_ts2(tDV, tR0 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), dom_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
+          }
           tc_commit(bar_do_empty + 8 * st);
-          // ---- S^T(T+1) (R0 is free: dV(T) was issued)
-          if (i + 1 < n_pairs) {
-            ok = issue_s(T + 1);
+          // ---- S^T(T+1) = K Q^T -> R0 (free: dV(T) was issued and the tensor pipe runs in order)
+          if (more) {
+            ok = need(have_q, bar_q_full + 8 * st1, par1, WAIT_BWD_QDO_FULL);
             if (!ok) break;
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) {
+              if (k == D / 16 - 2) have_ds = mbar_test(bar_ds_ready, T & 1);
+              mma_ss2(tR0, kk_lo + kstep_kmajor(k), qk1_lo + kstep_kmajor(k), IDESC_ST, k > 0);
+            }
+            tc_commit(bar_s_full);
           }
           // ---- dK += dS^T(T) Q(T)
-          ok = mbar_wait(bar_ds_ready, T & 1, ab, WAIT_BWD_PDS_FULL);
+          ok = need(have_ds, bar_ds_ready, T & 1, WAIT_BWD_PDS_FULL);
           if (!ok) break;
-          tc_fence_after();
+          have_do = false;
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
+          for (int k = 0; k < 8; ++k) {
+            if (k == 6) have_do = more && mbar_test(bar_do_full + 8 * st1, par1);
             mma_ts2(tDK, tR1 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), qm_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
+          }
           tc_commit(bar_q_empty + 8 * st);
         }
         if (!ok) break;

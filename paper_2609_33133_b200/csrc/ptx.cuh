@@ -44,6 +44,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// Non-blocking look at a phase.  The MMA-issuing thread calls it between the last MMAs of a group for the
+// barrier its next group needs: the tensor pipe queues only about two instructions, so a wait that sits
+// between two groups drains it, while a look that succeeds under the tail of the running group costs nothing.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
 
 // Shared per-CTA abort flag + global status word.  Every wait in the kernels
 // goes through mbar_wait: it spins on try_wait, and gives up when the abort
