@@ -3,13 +3,15 @@
 // shared prompt KV followed by a causal range of the query's own sequence
 // (Eq. 1); the online-softmax state (m, l, O_acc) of Sec. 3.3 is carried across
 // all of the item's KV tiles, which merges the two parts' partial states as it
-// goes.  The two query tiles of an item share every K/V tile the CTA loads, and
-// each has its own softmax warpgroup, so that one tile's exponentials overlap
-// the other tile's MMAs.
+// goes.  The two query tiles of an item share every K/V tile the CTA loads.
 //
-// Warp roles (320 threads): warps 0-3 own the rows of query tile 0, warps 4-7 the
-// rows of query tile 1 (a thread per row: softmax, O rescale, epilogue); warp 8
-// lane 0 issues TMA loads; warp 9 lane 0 issues tcgen05 MMAs.
+// Warp roles (320 threads): warps 0-7 are the softmax warps, warp 8 lane 0 issues
+// TMA loads, warp 9 issues tcgen05 MMAs (whole warp in lockstep, one elected lane).
+// All eight softmax warps work on ONE query tile at a time, two threads per row
+// (thread (w, lane) and (w + 4, lane) share row 32 (w % 4) + lane and take 64 key
+// columns each), and alternate between the two tiles.  What bounds a KV step is the
+// loop  softmax_g -> PV_g -> S_g(next) -> softmax_g  of one tile, so the softmax of a
+// tile has to be short; the other tile's MMAs run under it.
 // TMEM: S/P of tile 0 at column 0, of tile 1 at 128; O of tile 0 at 256, of tile 1 at 384.
 // MMA issue order per KV tile j: PV0(j), S0(j+1), PV1(j), S1(j+1).
 #pragma once
@@ -42,7 +44,8 @@ struct FwdSmem {
   static constexpr int kOffQ = 0;                       // two query tiles
   static constexpr int kOffKV = 2 * kTileBytes;         // [kStages]
   static constexpr int kOffBar = kOffKV + kStages * kTileBytes;
-  static constexpr int kBytes = kOffBar + 256;
+  static constexpr int kOffXch = kOffBar + 256;  // float [2][128][2]: row maxima / sums of the two column halves
+  static constexpr int kBytes = kOffXch + 2048;
 };
 
 template <int D>
@@ -66,6 +69,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   const uint32_t bar_kv_full = bars + 16, bar_kv_empty = bars + 48;  // [NS <= 4] each
   const uint32_t bar_s_full = bars + 80, bar_p_full = bars + 96;     // [2] each: per query tile
   const uint32_t bar_o_full = bars + 112, bar_o_empty = bars + 128;  // [2] each
+  const uint32_t bar_pair = bars + 160;                              // [4]: the two warps of a row quadrant
   volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_raw + SM::kOffBar + 144);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + SM::kOffBar + 152);
 
@@ -74,9 +78,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     mbar_init(bar_q_full, 1); mbar_init(bar_q_empty, 1);
     for (int s = 0; s < NS; ++s) { mbar_init(bar_kv_full + 8 * s, 1); mbar_init(bar_kv_empty + 8 * s, 1); }
     for (int g = 0; g < 2; ++g) {
-      mbar_init(bar_s_full + 8 * g, 1); mbar_init(bar_p_full + 8 * g, 4);
-      mbar_init(bar_o_full + 8 * g, 1); mbar_init(bar_o_empty + 8 * g, 4);
+      mbar_init(bar_s_full + 8 * g, 1); mbar_init(bar_p_full + 8 * g, 8);
+      mbar_init(bar_o_full + 8 * g, 1); mbar_init(bar_o_empty + 8 * g, 8);
     }
+    for (int q = 0; q < 4; ++q) mbar_init(bar_pair + 8 * q, 2);
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -126,88 +131,144 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     }
   } else if (warp == 9) {
     // -------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    // The whole warp walks the loops in lockstep and one elected lane issues: all the values that go into
+    // the descriptors are then warp-uniform (item fields come through a lane-0 broadcast), which keeps the
+    // instruction count per MMA small.  That matters because this warp shares its scheduler with two
+    // softmax warps, and a tensor pipe that queues only about two MMAs starves as soon as the issue of the
+    // next one is late.
+    {
       constexpr uint32_t IDESC_S = make_idesc(128, 128, 0, 0);
       constexpr uint32_t IDESC_PV = make_idesc(128, D, 0, 1);
+      const bool elected = elect_one();
+      const int it_b = __shfl_sync(0xffffffffu, it_begin, 0), it_e = __shfl_sync(0xffffffffu, it_end, 0);
       uint32_t kvc = 0, ic = 0, T = 0;
       bool ok = true;
-      const uint32_t q_lo[2] = {sdesc_lo(sQ, 16), sdesc_lo(sQ + TILE, 16)};
-      for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
+      const uint32_t q_lo0 = sdesc_lo(sQ, 16), q_lo1 = sdesc_lo(sQ + TILE, 16);
+      // a look that succeeded makes the wait unnecessary (every lane sees the same barrier state)
+      auto need = [&](bool have, uint32_t bar, uint32_t par, int site) -> bool {
+        if (!have && !mbar_spin(bar, par, ab, site)) return false;
+        tc_fence_after();
+        return true;
+      };
+      // K/V tiles of a KV step (V_j and K_{j+1}): waited for at the end of the step before, when this warp
+      // would otherwise only be waiting for the next P, so that the path from "P is there" to "PV issued"
+      // holds nothing but the P barrier
+      uint32_t vslot = 0, kslot = 0;
+      bool more = false;
+      auto acquire_kv = [&](int j, int n) -> bool {
+        vslot = kvc % NS;
+        if (!mbar_wait(bar_kv_full + 8 * vslot, (kvc / NS) & 1, ab, WAIT_FWD_KV_FULL)) return false;
+        ++kvc;
+        more = j + 1 < n;
+        if (more) {
+          kslot = kvc % NS;
+          if (!mbar_wait(bar_kv_full + 8 * kslot, (kvc / NS) & 1, ab, WAIT_FWD_KV_FULL)) return false;
+          ++kvc;
+        }
+        return true;
+      };
+      for (int it = it_b; it < it_e && ok; ++it, ++ic) {
         const int32_t *I = p.items + (size_t)it * 12;
-        const int n = ((I[5] + 127) >> 7) + ((I[7] + 127) >> 7);
+        const int n = __shfl_sync(0xffffffffu, ((I[5] + 127) >> 7) + ((I[7] + 127) >> 7), 0);
         ok = mbar_wait(bar_q_full, ic & 1, ab, WAIT_FWD_Q_FULL);
         if (!ok) break;
-        // S_g = Q_g K^T for both query tiles against the K tile in `slot`
-        auto issue_s = [&](uint32_t slot) {
-          const uint32_t k_lo = sdesc_lo(sKV + slot * TILE, 16);
-#pragma unroll
-          for (int g = 0; g < 2; ++g) {
-#pragma unroll
-            for (int k = 0; k < D / 16; ++k) mma_ss2(tmem + g * 128, q_lo[g] + kstep_kmajor(k), k_lo + kstep_kmajor(k), IDESC_S, k > 0);
-            tc_commit(bar_s_full + 8 * g);
-          }
-        };
+        bool have_p0 = false;
         {  // prologue: S0(0), S1(0)
           const uint32_t slot = kvc % NS;
-          ok = mbar_wait(bar_kv_full + 8 * slot, (kvc / NS) & 1, ab, WAIT_FWD_KV_FULL);
+          ok = need(false, bar_kv_full + 8 * slot, (kvc / NS) & 1, WAIT_FWD_KV_FULL);
           if (!ok) break;
-          tc_fence_after();
-          issue_s(slot);
-          tc_commit(bar_kv_empty + 8 * slot);
-          ++kvc;
-          if (n == 1) tc_commit(bar_q_empty);
-        }
-        for (int j = 0; j < n && ok; ++j, ++T) {
-          const uint32_t vslot = kvc % NS;
-          ok = mbar_wait(bar_kv_full + 8 * vslot, (kvc / NS) & 1, ab, WAIT_FWD_KV_FULL);
-          if (!ok) break;
-          ++kvc;
-          uint32_t kslot = 0;
-          const bool more = j + 1 < n;
-          if (more) {
-            kslot = kvc % NS;
-            ok = mbar_wait(bar_kv_full + 8 * kslot, (kvc / NS) & 1, ab, WAIT_FWD_KV_FULL);
-            if (!ok) break;
-            ++kvc;
+          const uint32_t k_lo = sdesc_lo(sKV + slot * TILE, 16);
+          if (elected) {
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) mma_ss2(tmem, q_lo0 + kstep_kmajor(k), k_lo + kstep_kmajor(k), IDESC_S, k > 0);
+            tc_commit(bar_s_full);
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) mma_ss2(tmem + 128, q_lo1 + kstep_kmajor(k), k_lo + kstep_kmajor(k), IDESC_S, k > 0);
+            tc_commit(bar_s_full + 8);
+            tc_commit(bar_kv_empty + 8 * slot);
+            if (n == 1) tc_commit(bar_q_empty);
           }
+          ++kvc;
+        }
+        ok = acquire_kv(0, n);
+        for (int j = 0; j < n && ok; ++j, ++T) {
           const uint32_t v_lo = sdesc_lo(sKV + vslot * TILE, 16384);
           const uint32_t k_lo = sdesc_lo(sKV + kslot * TILE, 16);
           const uint32_t acc0 = j > 0 ? 1u : 0u;
-#pragma unroll
-          for (int g = 0; g < 2; ++g) {
-            // PV_g(j): P_g (bf16, over S_g) times V
-            ok = mbar_wait(bar_p_full + 8 * g, T & 1, ab, WAIT_FWD_P_FULL);
+          // ---- query tile 0: PV0(j), then S0(j+1) over P0(j) (the tensor pipe runs in order)
+          ok = need(have_p0, bar_p_full, T & 1, WAIT_FWD_P_FULL);
+          if (!ok) break;
+          if (j == 0 && ic > 0) {
+            ok = need(false, bar_o_empty, (ic - 1) & 1, WAIT_FWD_O_EMPTY);
             if (!ok) break;
-            if (j == 0 && ic > 0) {
-              ok = mbar_wait(bar_o_empty + 8 * g, (ic - 1) & 1, ab, WAIT_FWD_O_EMPTY);
-              if (!ok) break;
-            }
-            tc_fence_after();
+          }
+          if (elected) {
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
-              mma_ts2(tmem + 256 + g * 128, tmem + g * 128 + k * 8, v_lo + kstep_mnmajor(k), IDESC_PV, acc0 | (uint32_t)(k > 0));
-            tc_commit(bar_o_full + 8 * g);
-            if (g == 1) tc_commit(bar_kv_empty + 8 * vslot);
-            // S_g(j+1) overwrites P_g(j): the tensor pipe runs in order
-            if (more) {
+            for (int k = 0; k < 8; ++k) mma_ts2(tmem + 256, tmem + k * 8, v_lo + kstep_mnmajor(k), IDESC_PV, acc0 | (uint32_t)(k > 0));
+            tc_commit(bar_o_full);
+          }
+          bool have_p1 = false;
+          if (more) {
+            if (elected) {
 #pragma unroll
-              for (int k = 0; k < D / 16; ++k) mma_ss2(tmem + g * 128, q_lo[g] + kstep_kmajor(k), k_lo + kstep_kmajor(k), IDESC_S, k > 0);
-              tc_commit(bar_s_full + 8 * g);
-              if (g == 1) {
-                tc_commit(bar_kv_empty + 8 * kslot);
-                if (j + 2 == n) tc_commit(bar_q_empty);
-              }
+              for (int k = 0; k < D / 16 - 2; ++k) mma_ss2(tmem, q_lo0 + kstep_kmajor(k), k_lo + kstep_kmajor(k), IDESC_S, k > 0);
             }
+            have_p1 = mbar_test(bar_p_full + 8, T & 1);
+            if (elected) {
+#pragma unroll
+              for (int k = D / 16 - 2; k < D / 16; ++k) mma_ss2(tmem, q_lo0 + kstep_kmajor(k), k_lo + kstep_kmajor(k), IDESC_S, k > 0);
+              tc_commit(bar_s_full);
+            }
+          }
+          // ---- query tile 1
+          ok = need(have_p1, bar_p_full + 8, T & 1, WAIT_FWD_P_FULL);
+          if (!ok) break;
+          if (j == 0 && ic > 0) {
+            ok = need(false, bar_o_empty + 8, (ic - 1) & 1, WAIT_FWD_O_EMPTY);
+            if (!ok) break;
+          }
+          if (elected) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) mma_ts2(tmem + 384, tmem + 128 + k * 8, v_lo + kstep_mnmajor(k), IDESC_PV, acc0 | (uint32_t)(k > 0));
+            tc_commit(bar_o_full + 8);
+            tc_commit(bar_kv_empty + 8 * vslot);
+          }
+          have_p0 = false;
+          if (more) {
+            if (elected) {
+#pragma unroll
+              for (int k = 0; k < D / 16 - 2; ++k) mma_ss2(tmem + 128, q_lo1 + kstep_kmajor(k), k_lo + kstep_kmajor(k), IDESC_S, k > 0);
+            }
+            have_p0 = mbar_test(bar_p_full, (T + 1) & 1);
+            if (elected) {
+#pragma unroll
+              for (int k = D / 16 - 2; k < D / 16; ++k) mma_ss2(tmem + 128, q_lo1 + kstep_kmajor(k), k_lo + kstep_kmajor(k), IDESC_S, k > 0);
+              tc_commit(bar_s_full + 8);
+              tc_commit(bar_kv_empty + 8 * kslot);
+              if (j + 2 == n) tc_commit(bar_q_empty);
+            }
+            ok = acquire_kv(j + 1, n);
           }
         }
       }
     }
   } else {
     // ------------------------------------------------- softmax / epilogue warps
-    const int g = warp >> 2;                 // query tile of the pair
-    const int r = (warp & 3) * 32 + lane;    // row inside the tile == TMEM lane
-    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tS = tmem + lane_off + g * 128, tO = tmem + lane_off + 256 + g * 128;
+    const int q4 = warp & 3, hl = warp >> 2;   // TMEM lane quadrant, column half
+    const int r = q4 * 32 + lane;              // row inside a query tile == TMEM lane
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    float *xch = reinterpret_cast<float *>(smem_raw + SM::kOffXch);
+    // exchange between the two threads of a row: write mine, meet the partner warp, read theirs
+    uint32_t xc = 0;
+    // (an mbarrier of count 2 rather than a named barrier: its wait is bounded like every other)
+    auto exchange = [&](float mine, bool &good) -> float {
+      float *buf = xch + (xc & 1) * 256 + r * 2;
+      buf[hl] = mine;
+      warp_arrive(bar_pair + 8 * q4);
+      good = mbar_wait(bar_pair + 8 * q4, xc & 1, ab, WAIT_FWD_PAIR);
+      ++xc;
+      return buf[hl ^ 1];
+    };
     uint32_t ic = 0, T = 0;
     bool ok = true;
     for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
@@ -215,125 +276,131 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const int q_tok0 = I[0], q_pos0 = I[1], q_rows = I[2], head = I[3], a_len = I[5], b_len = I[7];
       const int split = I[8], n_splits = I[9];
       const int nA = (a_len + 127) >> 7, n = nA + ((b_len + 127) >> 7);
-      const int my_pos = q_pos0 + g * 128 + r;  // position of this row in its sequence
-      float m_used = 0.f, l = 0.f;
-      for (int j = 0; j < n; ++j, ++T) {
-        ok = mbar_wait(bar_s_full + 8 * g, T & 1, ab, WAIT_FWD_S_FULL);
-        if (!ok) break;
-        tc_fence_after();
-        // number of leading key columns of this tile that the row sees
-        const int limit = (j < nA) ? (a_len - j * 128) : (my_pos + 1 - (j - nA) * 128);
-        // pass 1: row maximum of the raw scores (the scale is positive, so it commutes with the maximum);
-        // 64 columns per TMEM round trip
-        float mx = -INFINITY;
+      float m_used[2] = {0.f, 0.f}, l[2] = {0.f, 0.f};  // l: sum over this thread's columns only
+      for (int j = 0; j < n && ok; ++j, ++T) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          uint32_t sv[64];
-          tmem_ld32(tS + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
-          tmem_ld32(tS + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+        for (int g = 0; g < 2; ++g) {
+          const uint32_t tS = tmem + lane_off + g * 128, tO = tmem + lane_off + 256 + g * 128;
+          ok = mbar_wait(bar_s_full + 8 * g, T & 1, ab, WAIT_FWD_S_FULL);
+          if (!ok) break;
+          tc_fence_after();
+          // number of leading key columns of this KV tile that the row sees
+          const int limit = (j < nA) ? (a_len - j * 128) : (q_pos0 + g * 128 + r + 1 - (j - nA) * 128);
+          uint32_t s[64];  // raw scores of columns 64 hl .. 64 hl + 63
+          tmem_ld32(tS + hl * 64, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+          tmem_ld32(tS + hl * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
           tc_wait_ld();
-          if (limit >= 128) {
-#pragma unroll
-            for (int i = 0; i < 64; ++i) mx = fmaxf(mx, __uint_as_float(sv[i]));
-          } else {
+          if (limit < 128) {
 #pragma unroll
             for (int i = 0; i < 64; ++i)
-              if (h * 64 + i < limit) mx = fmaxf(mx, __uint_as_float(sv[i]));
+              if (hl * 64 + i >= limit) s[i] = 0xff800000u;  // -inf: exponentiates to zero
           }
-        }
-        mx *= p.scale_log2;
-        if (j == 0) {
-          m_used = (mx == -INFINITY) ? 0.f : mx;
-        } else {
-          const bool need = mx > m_used + kRescaleThreshold;
-          if (__any_sync(0xffffffffu, need)) {
-            ok = mbar_wait(bar_o_full + 8 * g, (T - 1) & 1, ab, WAIT_FWD_O_FULL);  // PV_g(j-1) done
-            if (!ok) break;
-            tc_fence_after();
-            float alpha = 1.f;
-            if (need) { alpha = ex2(m_used - mx); m_used = mx; l *= alpha; }
+          // row maximum of the raw scores (the scale is positive, so it commutes with the maximum)
+          float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-              uint32_t o[32];
-              tmem_ld32(tO + c * 32, o);
-              tc_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-              tmem_st32(tO + c * 32, o);
-            }
+          for (int i = 0; i < 64; i += 4) {
+            mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+            mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
           }
-        }
-        // pass 2: P = exp2(s * scale - m) from a second read of S; P (bf16) overwrites S columns
-        // [16c, 16c+16), which lie inside the columns [0, 32c+32) this thread has already consumed
-        float sum = 0.f;
-        uint32_t sa[32], sb[32];  // the next 32 columns are in flight while the current ones are exponentiated
-        tmem_ld32(tS, sa);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t (&cur)[32] = (c & 1) ? sb : sa;
-          uint32_t (&nxt)[32] = (c & 1) ? sa : sb;
-          tc_wait_ld();
-          if (c < 3) tmem_ld32(tS + (c + 1) * 32, nxt);
-          uint32_t pk[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float p0 = ex2(fmaf(__uint_as_float(cur[2 * i]), p.scale_log2, -m_used));
-            float p1 = ex2(fmaf(__uint_as_float(cur[2 * i + 1]), p.scale_log2, -m_used));
-            if (limit < 128) {
-              if (c * 32 + 2 * i >= limit) p0 = 0.f;
-              if (c * 32 + 2 * i + 1 >= limit) p1 = 0.f;
-            }
-            sum += p0 + p1;
-            pk[i] = pack_bf16(p0, p1);
-          }
-          tmem_st16(tS + c * 16, pk);
-        }
-        l += sum;
-        tc_wait_st();
-        tc_fence_before();
-        warp_arrive(bar_p_full + 8 * g);
-      }
-      if (!ok) break;
-      // ---- epilogue: O / l, LSE = ln2 * (m + log2 l)
-      ok = mbar_wait(bar_o_full + 8 * g, (T - 1) & 1, ab, WAIT_FWD_O_FULL);
-      if (!ok) break;
-      tc_fence_after();
-      const float inv_l = 1.f / l;
-      const long long tok = (long long)q_tok0 + g * 128 + r;
-      const bool valid = g * 128 + r < q_rows;
-      const float lse = (m_used + log2f(l)) * 0.6931471805599453f;
-#pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t o[32];
-        tmem_ld32(tO + c * 32, o);
-        tc_wait_ld();
-        if (valid) {
-          if (n_splits == 1) {
-            uint4 *dst = reinterpret_cast<uint4 *>(p.o + (tok * p.h_q + head) * D + c * 32);
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              uint4 w;
-              w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv_l, __uint_as_float(o[8 * v + 1]) * inv_l);
-              w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv_l, __uint_as_float(o[8 * v + 3]) * inv_l);
-              w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv_l, __uint_as_float(o[8 * v + 5]) * inv_l);
-              w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv_l, __uint_as_float(o[8 * v + 7]) * inv_l);
-              dst[v] = w;
-            }
+          mx0 = fmaxf(mx0, mx1);
+          // (the partner has loaded its scores before it gets here, so P may be stored over them below)
+          const float mx = fmaxf(mx0, exchange(mx0, ok)) * p.scale_log2;
+          if (!ok) break;
+          if (j == 0) {
+            m_used[g] = (mx == -INFINITY) ? 0.f : mx;
           } else {
-            float4 *dst = reinterpret_cast<float4 *>(p.part_o + (((long long)split * p.n_tok + tok) * p.h_q + head) * D + c * 32);
+            const bool need = mx > m_used[g] + kRescaleThreshold;
+            if (__any_sync(0xffffffffu, need)) {  // both warps of the row quadrant see the same rows
+              ok = mbar_wait(bar_o_full + 8 * g, (T - 1) & 1, ab, WAIT_FWD_O_FULL);  // PV_g(j-1) done
+              if (!ok) break;
+              tc_fence_after();
+              float alpha = 1.f;
+              if (need) { alpha = ex2(m_used[g] - mx); m_used[g] = mx; l[g] *= alpha; }
+#pragma unroll 1
+              for (int c = 0; c < D / 32; ++c) {  // this thread's half of the O row
+                uint32_t o[16];
+                tmem_ld16(tO + hl * (D / 2) + c * 16, o);
+                tc_wait_ld();
 #pragma unroll
-            for (int v = 0; v < 8; ++v)
-              dst[v] = make_float4(__uint_as_float(o[4 * v]) * inv_l, __uint_as_float(o[4 * v + 1]) * inv_l,
-                                   __uint_as_float(o[4 * v + 2]) * inv_l, __uint_as_float(o[4 * v + 3]) * inv_l);
+                for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                tmem_st16(tO + hl * (D / 2) + c * 16, o);
+              }
+            }
           }
+          // P = exp2(s * scale - m), bf16, stored over the S columns [32 hl + 16 c, +16).  One pair of
+          // columns in four takes its exponentials on the FMA pipe, the rest on the special-function unit.
+          float sum0 = 0.f, sum1 = 0.f;
+          const float mg = m_used[g];
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float x0 = fmaf(__uint_as_float(s[c * 32 + 2 * i]), p.scale_log2, -mg);
+              const float x1 = fmaf(__uint_as_float(s[c * 32 + 2 * i + 1]), p.scale_log2, -mg);
+              float p0, p1;
+              if ((i & 3) == 3) { p0 = ex2_fma(x0); p1 = ex2_fma(x1); }
+              else { p0 = ex2(x0); p1 = ex2(x1); }
+              sum0 += p0;
+              sum1 += p1;
+              pk[i] = pack_bf16(p0, p1);
+            }
+            tmem_st16(tS + hl * 32 + c * 16, pk);
+          }
+          l[g] += sum0 + sum1;
+          tc_wait_st();
+          tc_fence_before();
+          warp_arrive(bar_p_full + 8 * g);
         }
       }
-      if (valid) {
-        if (n_splits == 1) p.lse[(long long)head * p.n_tok + tok] = lse;
-        else p.part_lse[((long long)split * p.h_q + head) * p.n_tok + tok] = lse;
+      if (!ok) break;
+      // ---- epilogue: O / l, LSE = ln2 * (m + log2 l); each thread writes its half of the row
+#pragma unroll
+      for (int g = 0; g < 2; ++g) {
+        const uint32_t tO = tmem + lane_off + 256 + g * 128;
+        const float lt = l[g] + exchange(l[g], ok);
+        if (!ok) break;
+        ok = mbar_wait(bar_o_full + 8 * g, (T - 1) & 1, ab, WAIT_FWD_O_FULL);
+        if (!ok) break;
+        tc_fence_after();
+        const float inv_l = 1.f / lt;
+        const long long tok = (long long)q_tok0 + g * 128 + r;
+        const bool valid = g * 128 + r < q_rows;
+        constexpr int HALF = D / 2;
+#pragma unroll
+        for (int c = 0; c < HALF / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(tO + hl * HALF + c * 32, o);
+          tc_wait_ld();
+          if (valid) {
+            if (n_splits == 1) {
+              uint4 *dst = reinterpret_cast<uint4 *>(p.o + (tok * p.h_q + head) * D + hl * HALF + c * 32);
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                uint4 w;
+                w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv_l, __uint_as_float(o[8 * v + 1]) * inv_l);
+                w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv_l, __uint_as_float(o[8 * v + 3]) * inv_l);
+                w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv_l, __uint_as_float(o[8 * v + 5]) * inv_l);
+                w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv_l, __uint_as_float(o[8 * v + 7]) * inv_l);
+                dst[v] = w;
+              }
+            } else {
+              float4 *dst = reinterpret_cast<float4 *>(p.part_o + (((long long)split * p.n_tok + tok) * p.h_q + head) * D + hl * HALF + c * 32);
+#pragma unroll
+              for (int v = 0; v < 8; ++v)
+                dst[v] = make_float4(__uint_as_float(o[4 * v]) * inv_l, __uint_as_float(o[4 * v + 1]) * inv_l,
+                                     __uint_as_float(o[4 * v + 2]) * inv_l, __uint_as_float(o[4 * v + 3]) * inv_l);
+            }
+          }
+        }
+        if (valid && hl == 0) {
+          const float lse = (m_used[g] + log2f(lt)) * 0.6931471805599453f;
+          if (n_splits == 1) p.lse[(long long)head * p.n_tok + tok] = lse;
+          else p.part_lse[((long long)split * p.h_q + head) * p.n_tok + tok] = lse;
+        }
+        tc_fence_before();
+        warp_arrive(bar_o_empty + 8 * g);
       }
-      tc_fence_before();
-      warp_arrive(bar_o_empty + 8 * g);
     }
   }
 

@@ -10,7 +10,7 @@ namespace augtree {
 enum WaitSite : int {
   WAIT_NONE = 0,
   WAIT_FWD_Q_FULL = 1, WAIT_FWD_Q_EMPTY = 2, WAIT_FWD_KV_FULL = 3, WAIT_FWD_KV_EMPTY = 4, WAIT_FWD_S_FULL = 5,
-  WAIT_FWD_P_FULL = 6, WAIT_FWD_O_FULL = 7, WAIT_FWD_O_EMPTY = 8,
+  WAIT_FWD_P_FULL = 6, WAIT_FWD_O_FULL = 7, WAIT_FWD_O_EMPTY = 8, WAIT_FWD_PAIR = 9,
   WAIT_BWD_KV_FULL = 20, WAIT_BWD_KV_EMPTY = 21, WAIT_BWD_QDO_FULL = 22, WAIT_BWD_QDO_EMPTY = 23, WAIT_BWD_S_FULL = 24,
   WAIT_BWD_PDS_FULL = 25, WAIT_BWD_MMA2 = 26, WAIT_BWD_DQ_FREE = 27, WAIT_BWD_ACC_FULL = 28, WAIT_BWD_ACC_EMPTY = 29, WAIT_BWD_ROWS = 30,
   WAIT_DRAIN = 40
@@ -75,6 +75,25 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0) {
+      if (*ab.flag) return false;
+      if (clock64() - t0 > kWaitBudgetClocks) {
+        *ab.flag = 1;
+        if (atomicCAS(ab.status, 0, -5) == 0) ab.status[1] = site;
+        return false;
+      }
+    }
+  }
+}
+
+// The same wait as a pure spin on test_wait: for hand-offs on the critical path, where the time try_wait
+// takes to resume a suspended warp would be paid on every tile.
+__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity, const AbortCtx &ab, int site) {
+  if (mbar_test(bar, parity)) return true;
+  const long long t0 = clock64();
+  unsigned spins = 0;
+  while (true) {
+    if (mbar_test(bar, parity)) return true;
+    if ((++spins & 1023u) == 0) {
       if (*ab.flag) return false;
       if (clock64() - t0 > kWaitBudgetClocks) {
         *ab.flag = 1;
@@ -203,6 +222,11 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
                ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
@@ -233,6 +257,32 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+// True in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one() {
+  uint32_t e;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(e));
+  return e != 0;
+}
+// max(a, b, c) in one instruction (the two-input form issues at the same half rate)
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// 2^x on the FMA and integer pipes, for the share of the exponentials that the 4-per-clock special-function
+// unit would otherwise hold up: x = n + f with n = round(x) taken from the low mantissa bits of x + 1.5 * 2^23,
+// 2^f on [-0.5, 0.5] by a degree-4 polynomial (relative error 2.7e-6, far below the bf16 rounding of P), and
+// 2^n added into the exponent field.  x <= 0 up to the rescale threshold here; x < -125 returns 2^-125.
+__device__ __forceinline__ float ex2_fma(float x) {
+  x = fmaxf(x, -125.f);
+  const float t = x + 12582912.f;
+  const float f = x - (t - 12582912.f);
+  float p = fmaf(f, 0.009570036083459854f, 0.05591771379113197f);
+  p = fmaf(p, f, 0.240247443318367f);
+  p = fmaf(p, f, 0.6931218504905701f);
+  p = fmaf(p, f, 0.9999992847442627f);
+  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
 }
 __device__ __forceinline__ void red_add_v4(float *gptr, float a, float b, float c, float d) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(gptr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
