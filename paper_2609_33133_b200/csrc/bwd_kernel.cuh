@@ -152,21 +152,25 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     }
   } else if (warp == 9) {
     // -------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    // The whole warp runs the loops in lockstep and one elected lane issues (warp-uniform descriptor
+    // arithmetic: few instructions per MMA, which matters next to two busy element-wise warps on the same
+    // scheduler).  Each group looks at the barrier of the group after it before its own last two MMAs
+    // (`have`), so that a hand-off which has already happened costs the tensor pipe nothing.
+    {
       constexpr uint32_t IDESC_ST = make_idesc(128, 128, 0, 0);  // S^T, dP^T: both operands K-major
       constexpr uint32_t IDESC_ACC = make_idesc(128, D, 0, 1);   // dV, dK: A from TMEM, B = dO / Q MN-major
+      constexpr int NK = D / 16;
+      const bool elected = elect_one();
+      const int it_b = __shfl_sync(0xffffffffu, it_begin, 0), it_e = __shfl_sync(0xffffffffu, it_end, 0);
       uint32_t ic = 0, T = 0;
       bool ok = true;
       const uint32_t kk_lo = sdesc_lo(sK, 16), vk_lo = sdesc_lo(sV, 16);
-      // Each group looks at the barrier of the group after it before its own last two MMAs (`have`), so
-      // that a hand-off which has already happened costs the tensor pipe nothing; only a look that fails
-      // turns into a wait between the groups.
       auto need = [&](bool have, uint32_t bar, uint32_t par, int site) -> bool {
         if (!have && !mbar_wait(bar, par, ab, site)) return false;
         tc_fence_after();
         return true;
       };
-      for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
+      for (int it = it_b; it < it_e && ok; ++it, ++ic) {
         const int32_t *I = p.items + (size_t)it * 8;
         const int kv_pos0 = I[1], mode = I[4], seg0 = I[5], nseg = I[6];
         int n_pairs = 0;
@@ -174,6 +178,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           const int nqt = (p.segs[3 * sg + 1] + 127) >> 7;
           n_pairs += (nqt - (mode ? 0 : (kv_pos0 >> 7))) * rep;
         }
+        n_pairs = __shfl_sync(0xffffffffu, n_pairs, 0);
         ok = mbar_wait(bar_kv_full, ic & 1, ab, WAIT_BWD_KV_FULL);
         if (!ok) break;
         bool have_do = false;
@@ -182,12 +187,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           ok = need(false, bar_q_full + 8 * st, par, WAIT_BWD_QDO_FULL);
           if (!ok) break;
           const uint32_t qk_lo = sdesc_lo(sQ0 + st * TILE, 16);
-#pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            if (k == D / 16 - 2) have_do = mbar_test(bar_do_full + 8 * st, par);
-            mma_ss2(tR0, kk_lo + kstep_kmajor(k), qk_lo + kstep_kmajor(k), IDESC_ST, k > 0);
-          }
-          tc_commit(bar_s_full);
+          mma_group<NK>(elected,
+                        [&](int k) { mma_ss2(tR0, kk_lo + kstep_kmajor(k), qk_lo + kstep_kmajor(k), IDESC_ST, k > 0); },
+                        [&]() { have_do = mbar_test(bar_do_full + 8 * st, par); });
+          if (elected) tc_commit(bar_s_full);
         }
         for (int i = 0; i < n_pairs && ok; ++i, ++T) {
           const uint32_t st = T % NST, par = (T / NST) & 1;
@@ -200,12 +203,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           // ---- dP^T(T) = V dO^T -> R1
           ok = need(have_do, bar_do_full + 8 * st, par, WAIT_BWD_QDO_FULL);
           if (!ok) break;
-#pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            if (k == D / 16 - 2) have_p = mbar_test(bar_p_ready, T & 1);
-            mma_ss2(tR1, vk_lo + kstep_kmajor(k), dok_lo + kstep_kmajor(k), IDESC_ST, k > 0);
-          }
-          tc_commit(bar_dp_full);
+          mma_group<NK>(elected,
+                        [&](int k) { mma_ss2(tR1, vk_lo + kstep_kmajor(k), dok_lo + kstep_kmajor(k), IDESC_ST, k > 0); },
+                        [&]() { have_p = mbar_test(bar_p_ready, T & 1); });
+          if (elected) tc_commit(bar_dp_full);
           // ---- dV += P^T(T) dO(T)
           if (i == 0 && ic > 0) {  // the previous item's dV/dK must have left TMEM
             ok = mbar_wait(bar_acc_empty, (ic - 1) & 1, ab, WAIT_BWD_ACC_EMPTY);
@@ -213,37 +214,35 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           }
           ok = need(have_p, bar_p_ready, T & 1, WAIT_BWD_PDS_FULL);
           if (!ok) break;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {  // query columns 16k..16k+15: P^T sits at R0 columns 8k (k<4) or 64+8(k-4)
-            if (k == 6) have_q = more && mbar_test(bar_q_full + 8 * st1, par1);
-            mma_ts2(tDV, tR0 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), dom_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
-          }
-          tc_commit(bar_do_empty + 8 * st);
+          // (query columns 16k..16k+15: P^T sits at R0 columns 8k (k<4) or 64+8(k-4))
+          mma_group<8>(elected,
+                       [&](int k) {
+                         mma_ts2(tDV, tR0 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), dom_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
+                       },
+                       [&]() { have_q = more && mbar_test(bar_q_full + 8 * st1, par1); });
+          if (elected) tc_commit(bar_do_empty + 8 * st);
           // ---- S^T(T+1) = K Q^T -> R0 (free: dV(T) was issued and the tensor pipe runs in order)
           if (more) {
             ok = need(have_q, bar_q_full + 8 * st1, par1, WAIT_BWD_QDO_FULL);
             if (!ok) break;
-#pragma unroll
-            for (int k = 0; k < D / 16; ++k) {
-              if (k == D / 16 - 2) have_ds = mbar_test(bar_ds_ready, T & 1);
-              mma_ss2(tR0, kk_lo + kstep_kmajor(k), qk1_lo + kstep_kmajor(k), IDESC_ST, k > 0);
-            }
-            tc_commit(bar_s_full);
+            mma_group<NK>(elected,
+                          [&](int k) { mma_ss2(tR0, kk_lo + kstep_kmajor(k), qk1_lo + kstep_kmajor(k), IDESC_ST, k > 0); },
+                          [&]() { have_ds = mbar_test(bar_ds_ready, T & 1); });
+            if (elected) tc_commit(bar_s_full);
           }
           // ---- dK += dS^T(T) Q(T)
           ok = need(have_ds, bar_ds_ready, T & 1, WAIT_BWD_PDS_FULL);
           if (!ok) break;
           have_do = false;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            if (k == 6) have_do = more && mbar_test(bar_do_full + 8 * st1, par1);
-            mma_ts2(tDK, tR1 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), qm_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
-          }
-          tc_commit(bar_q_empty + 8 * st);
+          mma_group<8>(elected,
+                       [&](int k) {
+                         mma_ts2(tDK, tR1 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), qm_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
+                       },
+                       [&]() { have_do = more && mbar_test(bar_do_full + 8 * st1, par1); });
+          if (elected) tc_commit(bar_q_empty + 8 * st);
         }
         if (!ok) break;
-        tc_commit(bar_acc_full);
-        tc_commit(bar_kv_empty);
+        if (elected) { tc_commit(bar_acc_full); tc_commit(bar_kv_empty); }
       }
     }
   } else {

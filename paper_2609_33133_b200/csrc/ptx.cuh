@@ -264,6 +264,20 @@ __device__ __forceinline__ bool elect_one() {
   asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(e));
   return e != 0;
 }
+// One group of NK MMAs issued by the elected lane of a warp that runs in lockstep, with a look at the next
+// group's barrier (every lane) slipped in before the last two: mma(k) issues instruction k, look() is the test.
+template <int NK, class MmaK, class Look>
+__device__ __forceinline__ void mma_group(bool elected, MmaK mma, Look look) {
+  if (elected) {
+#pragma unroll
+    for (int k = 0; k < NK - 2; ++k) mma(k);
+  }
+  look();
+  if (elected) {
+#pragma unroll
+    for (int k = NK - 2; k < NK; ++k) mma(k);
+  }
+}
 // max(a, b, c) in one instruction (the two-input form issues at the same half rate)
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
