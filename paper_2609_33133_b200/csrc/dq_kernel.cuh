@@ -133,64 +133,82 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     }
   } else if (warp == 9) {
     // -------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    // The whole warp runs the loops in lockstep and one elected lane issues (warp-uniform descriptor
+    // arithmetic keeps the instruction count per MMA small next to two busy element-wise warps on the
+    // same scheduler); each group looks at the next group's barrier before its own last two MMAs.
+    {
       constexpr uint32_t IDESC_S = make_idesc(128, 128, 0, 0);  // S, dP: A from TMEM, B K-major
       constexpr uint32_t IDESC_DQ = make_idesc(128, D, 0, 1);   // dQ: A = dS from TMEM, B = K MN-major
+      constexpr int NKS = D / 16;
+      const bool elected = elect_one();
+      const int it_b = __shfl_sync(0xffffffffu, it_begin, 0), it_e = __shfl_sync(0xffffffffu, it_end, 0);
       uint32_t ic = 0, T = 0;
       bool ok = true;
-      auto issue_s = [&](uint32_t Tn) -> bool {  // S(Tn) = Q K^T
+      auto need = [&](bool have, uint32_t bar, uint32_t par, int site) -> bool {
+        if (!have && !mbar_wait(bar, par, ab, site)) return false;
+        tc_fence_after();
+        return true;
+      };
+      // S(Tn) = Q K^T; `look` runs before the last two MMAs
+      auto issue_s = [&](uint32_t Tn, bool have, auto look) -> bool {
         const uint32_t ks = Tn % NK;
-        if (!mbar_wait(bar_k_full + 8 * ks, (Tn / NK) & 1, ab, WAIT_DQ_K)) return false;
-        tc_fence_after();
+        if (!need(have, bar_k_full + 8 * ks, (Tn / NK) & 1, WAIT_DQ_K)) return false;
         const uint32_t k_lo = sdesc_lo(sK0 + ks * TILE, 16);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) mma_ts2(tS, tQ + k * 8, k_lo + kstep_kmajor(k), IDESC_S, k > 0);
-        tc_commit(bar_s_full);
+        mma_group<NKS>(elected, [&](int k) { mma_ts2(tS, tQ + k * 8, k_lo + kstep_kmajor(k), IDESC_S, k > 0); }, look);
+        if (elected) tc_commit(bar_s_full);
         return true;
       };
-      auto issue_dp = [&](uint32_t Tn) -> bool {  // dP(Tn) = dO V^T
+      // dP(Tn) = dO V^T
+      auto issue_dp = [&](uint32_t Tn, bool have, auto look) -> bool {
         const uint32_t vs = Tn % NV;
-        if (!mbar_wait(bar_v_full + 8 * vs, (Tn / NV) & 1, ab, WAIT_DQ_V)) return false;
-        tc_fence_after();
+        if (!need(have, bar_v_full + 8 * vs, (Tn / NV) & 1, WAIT_DQ_V)) return false;
         const uint32_t v_lo = sdesc_lo(sV0 + vs * TILE, 16);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) mma_ts2(tDP, tDO + k * 8, v_lo + kstep_kmajor(k), IDESC_S, k > 0);
-        tc_commit(bar_dp_full);
-        tc_commit(bar_v_empty + 8 * vs);
+        mma_group<NKS>(elected, [&](int k) { mma_ts2(tDP, tDO + k * 8, v_lo + kstep_kmajor(k), IDESC_S, k > 0); }, look);
+        if (elected) { tc_commit(bar_dp_full); tc_commit(bar_v_empty + 8 * vs); }
         return true;
       };
-      for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
+      for (int it = it_b; it < it_e && ok; ++it, ++ic) {
         const int32_t *I = p.items + (size_t)it * 12;
-        const int n = ((I[5] + 127) >> 7) + ((I[7] + 127) >> 7);
+        const int n = __shfl_sync(0xffffffffu, ((I[5] + 127) >> 7) + ((I[7] + 127) >> 7), 0);
         ok = mbar_wait(bar_qt_ready, ic & 1, ab, WAIT_DQ_QT);
         if (!ok) break;
-        ok = issue_s(T) && issue_dp(T);
+        bool have_sread = false, have_ds = false, have_v = false, have_k = false;
+        ok = issue_s(T, false, [&]() { have_v = mbar_test(bar_v_full + 8 * (T % NV), (T / NV) & 1); }) &&
+             issue_dp(T, have_v, [&]() { have_sread = n > 1 && mbar_test(bar_s_read, T & 1); });
         for (int i = 0; i < n && ok; ++i, ++T) {
-          if (i + 1 < n) {  // S(T+1): the warps must have read S(T) out of TMEM
-            ok = mbar_wait(bar_s_read, T & 1, ab, WAIT_DQ_SREAD);
+          const bool more = i + 1 < n;
+          have_ds = false;
+          if (more) {  // S(T+1): the warps must have read S(T) out of TMEM
+            ok = need(have_sread, bar_s_read, T & 1, WAIT_DQ_SREAD);
             if (!ok) break;
-            ok = issue_s(T + 1);
+            have_k = mbar_test(bar_k_full + 8 * ((T + 1) % NK), ((T + 1) / NK) & 1);
+            ok = issue_s(T + 1, have_k, [&]() { have_ds = mbar_test(bar_ds_ready, T & 1); });
             if (!ok) break;
           }
           // dQ += dS(T) K(T)
-          ok = mbar_wait(bar_ds_ready, T & 1, ab, WAIT_DQ_DS);
+          ok = need(have_ds, bar_ds_ready, T & 1, WAIT_DQ_DS);
           if (!ok) break;
           if (i == 0 && ic > 0) {  // the previous item's dQ must have left TMEM
-            ok = mbar_wait(bar_dq_empty, (ic - 1) & 1, ab, WAIT_DQ_EMPTY);
+            ok = need(false, bar_dq_empty, (ic - 1) & 1, WAIT_DQ_EMPTY);
             if (!ok) break;
           }
-          tc_fence_after();
           const uint32_t ks = T % NK;
           const uint32_t km_lo = sdesc_lo(sK0 + ks * TILE, 16384);
           const uint32_t acc0 = i > 0 ? 1u : 0u;
-#pragma unroll
-          for (int k = 0; k < 8; ++k)  // key columns 16k..16k+15: dS sits at dP columns 8k (k<4) or 64+8(k-4)
-            mma_ts2(tDQ, tDP + (k < 4 ? k * 8 : 64 + (k - 4) * 8), km_lo + kstep_mnmajor(k), IDESC_DQ, acc0 | (uint32_t)(k > 0));
-          tc_commit(bar_k_empty + 8 * ks);
-          if (i + 1 < n) ok = issue_dp(T + 1);  // overwrites dS(T): the tensor pipe runs in order
+          have_v = false;
+          // (key columns 16k..16k+15: dS sits at dP columns 8k (k<4) or 64+8(k-4))
+          mma_group<8>(elected,
+                       [&](int k) {
+                         mma_ts2(tDQ, tDP + (k < 4 ? k * 8 : 64 + (k - 4) * 8), km_lo + kstep_mnmajor(k), IDESC_DQ, acc0 | (uint32_t)(k > 0));
+                       },
+                       [&]() { have_v = more && mbar_test(bar_v_full + 8 * ((T + 1) % NV), ((T + 1) / NV) & 1); });
+          if (elected) tc_commit(bar_k_empty + 8 * ks);
+          have_sread = false;
+          if (more)  // dP(T+1) overwrites dS(T): the tensor pipe runs in order
+            ok = issue_dp(T + 1, have_v, [&]() { have_sread = i + 2 < n && mbar_test(bar_s_read, (T + 1) & 1); });
         }
         if (!ok) break;
-        tc_commit(bar_dq_full);
+        if (elected) tc_commit(bar_dq_full);
       }
     }
   } else {
