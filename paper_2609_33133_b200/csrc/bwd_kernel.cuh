@@ -274,7 +274,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         pr[i + 0] = ex2(fmaf(__uint_as_float(sv[i + 0]), p.scale_log2, -l4.x));
         pr[i + 1] = ex2(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -l4.y));
         pr[i + 2] = ex2(fmaf(__uint_as_float(sv[i + 2]), p.scale_log2, -l4.z));
-        pr[i + 3] = ex2(fmaf(__uint_as_float(sv[i + 3]), p.scale_log2, -l4.w));
+        pr[i + 3] = ex2_fma(fmaf(__uint_as_float(sv[i + 3]), p.scale_log2, -l4.w));  // one in four on the FMA pipe
       }
       if (!all_visible) {
 #pragma unroll

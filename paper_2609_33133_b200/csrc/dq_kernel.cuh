@@ -265,7 +265,10 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           const int limit = (i < nA) ? (a_len - i * 128) : (q_pos0 + r + 1 - (i - nA) * 128);
           const int lim = limit - ch * 64;
 #pragma unroll
-          for (int c = 0; c < 64; ++c) pr[c] = ex2(fmaf(__uint_as_float(sv[c]), p.scale_log2, -lse2));
+          for (int c = 0; c < 64; ++c) {  // one exponential in four on the FMA pipe, the rest on the special-function unit
+            const float x = fmaf(__uint_as_float(sv[c]), p.scale_log2, -lse2);
+            pr[c] = (c & 3) == 3 ? ex2_fma(x) : ex2(x);
+          }
           if (lim < 64) {
 #pragma unroll
             for (int c = 0; c < 64; ++c)
