@@ -66,6 +66,12 @@ def peaks():
     return {"bf16_tflops": FALLBACK_BF16_TFLOPS, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture of this workload (the summary under
+# profiles/ gives the command); None for workloads that were not captured
+NCU_DRAM_BYTES = {("cfg2-7b-layer", "replay_bwd_dkdv"): 1.226e9, ("cfg2-7b-layer", "replay_bwd_dq"): 0.384e9,
+                  ("cfg2-7b-layer", "replay_fwd"): 0.254e9}
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -281,7 +287,7 @@ def main():
     dom = max(per_kernel, key=lambda n: per_kernel[n]["ms"])
     roofline = {"bound": "tensor", "kernel": f"{kfun[dom]} ({dom})", "achieved": per_kernel[dom]["tflops"],
                 "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": per_kernel[dom]["tflops"] / pk["bf16_tflops"],
-                "peak_source": f"{pk['source']} cuBLAS bf16 burst", "traffic": None}
+                "peak_source": f"{pk['source']} cuBLAS bf16 burst", "traffic": NCU_DRAM_BYTES.get((w.name, dom))}
 
     # ---- end to end: pinned host inputs copied in, results copied out, every step
     host_in = {k: v.cpu().pin_memory() for k, v in t_dev.items()}

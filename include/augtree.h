@@ -101,7 +101,8 @@ enum {
 
 /*
  * Pack and schedule (host).  Validates the descriptor, builds the prefix sums
- * and, for each of the four kernels, the list of work items and their
+ * and, for each of the six schedules (forward, key-side and query-side
+ * backward, each for the prefill and the replay call), the list of work items and their
  * assignment to `n_lanes` replay lanes: items weighted by their valid Q-KV
  * tile count are placed largest first on the least loaded lane (the balanced
  * makespan assignment of Sec. 3.4, Eq. 6, in its greedy form with one round).
