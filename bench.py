@@ -196,22 +196,23 @@ def time_steps(step_fn, steps, warmup, dist, sampler_index=None):
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
     sampler = ClockSampler(sampler_index) if sampler_index is not None else None
     if sampler:
         sampler.__enter__()
         time.sleep(0.15)
-    e0.record()
-    for _ in range(steps):
+    ev[0].record()
+    for i in range(steps):
         step_fn()
-    e1.record()
+        ev[i + 1].record()
     torch.cuda.synchronize()
     if sampler:
         sampler.__exit__()
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    ms = max_over_ranks(e0.elapsed_time(e1), dist)
+    ms = max_over_ranks(ev[0].elapsed_time(ev[steps]), dist)
+    time_steps.per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]  # this rank's, for median / min
     return ms, (sampler.summary() if sampler else None)
 
 
@@ -256,8 +257,10 @@ def main():
     t_dev = wl.make_tensors(w, device="cuda" if big else "cpu")
     t_dev = {k: v.cuda() for k, v in t_dev.items()}
     splits = 4 if w.extra.get("force_split") else 0
+    t_plan = time.perf_counter()
     plan = B.Plan(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, device=local_rank, flags=B.FLAG_ZERO_PROMPT_GRAD,
                   kv_splits=splits)
+    plan_ms = (time.perf_counter() - t_plan) * 1e3  # pack and schedule on the host + table upload; not part of a step
     out = B.alloc_outputs(plan)
 
     def step():
@@ -274,6 +277,7 @@ def main():
     kt = [plan.kernel_time(k) for k in range(6)]
     plan.set_timing(False)
     ms_step = ms / args.steps
+    per_step = sorted(time_steps.per_step)
     value = aggregate_tflops(fl["total"], world, ms_step)
 
     # dominant kernel: the replay backward tile kernel
@@ -336,7 +340,8 @@ def main():
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "ms_per_step": ms_step, "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": per_step[0],
+            "plan_create_ms": plan_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
             "config": {"workload": w.name, "groups": w.n_groups, "prompt_tokens": w.total_prompt, "response_tokens": w.total_response,
                        "h_q": w.h_q, "h_kv": w.h_kv, "head_dim": w.head_dim, "useful_tflop_per_step": fl["total"] / 1e12,

@@ -84,3 +84,76 @@ def test_config2_full_size_sampled(B):
     assert np.abs(got1["dq_r"]).max() <= 0.05 and np.abs(got1["dk_p"]).max() <= 0.5
     # LSE does not depend on V
     assert np.array_equal(got1["lse_r"], got["lse_r"]) and np.array_equal(got1["lse_p"], got["lse_p"])
+
+
+class _DeviceRows:
+    """Indexable view of a device tensor that hands the oracle's row forms fp32 host copies of just the
+    slices they ask for (the full-size tensors of configurations 3-5 are too large to widen on the host)."""
+
+    def __init__(self, t):
+        self.t = t
+
+    def __getitem__(self, idx):
+        return self.t[idx].float().cpu().numpy()
+
+
+@pytest.mark.parametrize("index", [3, 4, 5])
+def test_large_configs_full_size_sampled(B, index):
+    """Configurations 3-5 at full size (0.15 M, 0.65 M and 0.94 M tokens; the query tensors of 4 and 5 have more
+    than 2^31 elements), in the plan bench.py times: sampled query rows and keys against the oracle's row forms,
+    among them the first and last tokens, tokens either side of element offset 2^31, and ends of branches."""
+    w = wl.config(index)
+    splits = 4 if w.extra.get("force_split") else 0
+    t = wl.make_tensors(w, device="cuda")
+    plan = B.Plan(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, device=0, flags=B.FLAG_ZERO_PROMPT_GRAD, kv_splits=splits)
+    out = B.alloc_outputs(plan)
+    B.run_forward_backward(plan, t, out)
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0)
+    tb = ora.TreeBatch(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim)
+    f = {k: _DeviceRows(v) for k, v in t.items()}
+    host = lambda x: x.float().cpu().numpy().astype(np.float64)
+    rng = np.random.default_rng(40 + index)
+    tp, tr = w.total_prompt, w.total_response
+    edge = 2 ** 31 // (w.h_q * w.head_dim)  # first token whose element offset in a query-sized tensor passes 2^31
+    rows = [("p", 0, 0), ("p", tp - 1, w.h_q - 1), ("r", 0, 1), ("r", tr - 1, w.h_q - 1)]
+    rows += [("r", tok, int(rng.integers(0, w.h_q))) for tok in (edge - 1, edge, edge + 1, 2 * edge) if tok < tr]
+    rows += [("p", int(rng.integers(0, tp)), int(rng.integers(0, w.h_q))) for _ in range(4)]
+    rows += [("r", int(rng.integers(0, tr)), int(rng.integers(0, w.h_q))) for _ in range(8)]
+    for kind, tok, h in rows:
+        o, lse = ora.forward_row(tb, f["q_p"], f["k_p"], f["v_p"], f["q_r"], f["k_r"], f["v_r"], kind, tok, h)
+        dq = ora.dq_row(tb, f["q_p"], f["k_p"], f["v_p"], f["do_p"], f["q_r"], f["k_r"], f["v_r"], f["do_r"], kind, tok, h)
+        sfx = "_p" if kind == "p" else "_r"
+        g_lse, g_o, g_dq = float(out["lse" + sfx][h, tok]), host(out["o" + sfx][tok, h]), host(out["dq" + sfx][tok, h])
+        assert abs(g_lse - lse) <= pu.LSE_ABS, (kind, tok, h)
+        assert np.abs(g_o - o).max() <= pu.MAX_ABS, (kind, tok, h)
+        assert np.linalg.norm(g_o - o) <= 2 * pu.REL_L2 * np.linalg.norm(o) + 1e-3, (kind, tok, h)
+        assert np.abs(g_dq - dq).max() <= pu.MAX_ABS, (kind, tok, h)
+        assert np.linalg.norm(g_dq - dq) <= 2 * pu.REL_L2 * np.linalg.norm(dq) + 1e-3, (kind, tok, h)
+    # response keys near the end of a branch (few rows see them): the last branch, one in the middle, the first
+    cu_r = tb.cu_r
+    for b in (len(cu_r) - 2, (len(cu_r) - 1) // 2, 0):
+        for back in (1, 9):
+            tok = int(cu_r[b + 1]) - back
+            if tok < int(cu_r[b]):
+                continue
+            c = int(rng.integers(0, w.h_kv))
+            dk, dv = ora.dkv_key(tb, f["q_p"], f["k_p"], f["v_p"], f["do_p"], f["q_r"], f["k_r"], f["v_r"], f["do_r"], "r", tok, c)
+            g_dk, g_dv = host(out["dk_r"][tok, c]), host(out["dv_r"][tok, c])
+            assert np.abs(g_dk - dk).max() <= pu.MAX_ABS and np.abs(g_dv - dv).max() <= pu.MAX_ABS, (b, tok, c)
+            assert np.linalg.norm(g_dv - dv) <= 2 * pu.REL_L2 * np.linalg.norm(dv) + 2e-3, (b, tok, c)
+    # a prompt key (Eq. 2: summed over every branch and query head of its group): the last prompt token of the
+    # group whose branches are shortest, so that the per-key oracle form stays affordable
+    cost = [sum(bl) * (p + max(bl)) for p, bl in zip(w.prompt_len, w.branch_len)]
+    g = int(np.argmin(cost))
+    if cost[g] * (w.h_q // w.h_kv) * w.head_dim <= 4e10:
+        tok = int(tb.cu_p[g + 1]) - 1
+        dk, dv = ora.dkv_key(tb, f["q_p"], f["k_p"], f["v_p"], f["do_p"], f["q_r"], f["k_r"], f["v_r"], f["do_r"], "p", tok, 0)
+        g_dk, g_dv = host(out["dk_p"][tok, 0]), host(out["dv_p"][tok, 0])
+        bound = max(pu.MAX_ABS, pu.BF16_UNIT_ROUNDOFF * max(np.abs(dk).max(), np.abs(dv).max()))
+        assert np.abs(g_dk - dk).max() <= bound and np.abs(g_dv - dv).max() <= bound, (g, tok)
+        assert np.linalg.norm(g_dv - dv) <= 2 * pu.REL_L2 * np.linalg.norm(dv) + 2e-3, (g, tok)
+    # every output finite (checked on the device)
+    for k, v in out.items():
+        if k != "ws":
+            assert bool(torch.isfinite(v).all()), k
