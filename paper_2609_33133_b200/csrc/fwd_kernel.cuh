@@ -7,11 +7,12 @@
 //
 // Warp roles (320 threads): warps 0-7 are the softmax warps, warp 8 lane 0 issues
 // TMA loads, warp 9 issues tcgen05 MMAs (whole warp in lockstep, one elected lane).
-// All eight softmax warps work on ONE query tile at a time, two threads per row
-// (thread (w, lane) and (w + 4, lane) share row 32 (w % 4) + lane and take 64 key
-// columns each), and alternate between the two tiles.  What bounds a KV step is the
-// loop  softmax_g -> PV_g -> S_g(next) -> softmax_g  of one tile, so the softmax of a
-// tile has to be short; the other tile's MMAs run under it.
+// All eight softmax warps work on ONE query tile at a time, 16 rows each, and
+// alternate between the two tiles.  They read S in the accumulator-fragment layout
+// (tcgen05.ld 16x256b): a row is spread over the four threads of a quad, so the row
+// maximum and sum are two shuffles and no warp waits for another.  What bounds a KV
+// step is the loop  softmax_g -> PV_g -> S_g(next) -> softmax_g  of one tile, so the
+// softmax of a tile has to be short; the other tile's MMAs run under it.
 // TMEM: S/P of tile 0 at column 0, of tile 1 at 128; O of tile 0 at 256, of tile 1 at 384.
 // MMA issue order per KV tile j: PV0(j), S0(j+1), PV1(j), S1(j+1).
 #pragma once
@@ -44,8 +45,7 @@ struct FwdSmem {
   static constexpr int kOffQ = 0;                       // two query tiles
   static constexpr int kOffKV = 2 * kTileBytes;         // [kStages]
   static constexpr int kOffBar = kOffKV + kStages * kTileBytes;
-  static constexpr int kOffXch = kOffBar + 256;  // float [2][128][2]: row maxima / sums of the two column halves
-  static constexpr int kBytes = kOffXch + 2048;
+  static constexpr int kBytes = kOffBar + 256;
 };
 
 template <int D>
@@ -69,7 +69,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   const uint32_t bar_kv_full = bars + 16, bar_kv_empty = bars + 48;  // [NS <= 4] each
   const uint32_t bar_s_full = bars + 80, bar_p_full = bars + 96;     // [2] each: per query tile
   const uint32_t bar_o_full = bars + 112, bar_o_empty = bars + 128;  // [2] each
-  const uint32_t bar_pair = bars + 160;                              // [4]: the two warps of a row quadrant
   volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_raw + SM::kOffBar + 144);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + SM::kOffBar + 152);
 
@@ -81,7 +80,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       mbar_init(bar_s_full + 8 * g, 1); mbar_init(bar_p_full + 8 * g, 8);
       mbar_init(bar_o_full + 8 * g, 1); mbar_init(bar_o_empty + 8 * g, 8);
     }
-    for (int q = 0; q < 4; ++q) mbar_init(bar_pair + 8 * q, 2);
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -254,20 +252,21 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     }
   } else {
     // ------------------------------------------------- softmax / epilogue warps
-    const int q4 = warp & 3, hl = warp >> 2;   // TMEM lane quadrant, column half
-    const int r = q4 * 32 + lane;              // row inside a query tile == TMEM lane
-    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
-    float *xch = reinterpret_cast<float *>(smem_raw + SM::kOffXch);
-    // exchange between the two threads of a row: write mine, meet the partner warp, read theirs
-    uint32_t xc = 0;
-    // (an mbarrier of count 2 rather than a named barrier: its wait is bounded like every other)
-    auto exchange = [&](float mine, bool &good) -> float {
-      float *buf = xch + (xc & 1) * 256 + r * 2;
-      buf[hl] = mine;
-      warp_arrive(bar_pair + 8 * q4);
-      good = mbar_wait(bar_pair + 8 * q4, xc & 1, ab, WAIT_FWD_PAIR);
-      ++xc;
-      return buf[hl ^ 1];
+    // Warp w works on 16 rows of the current query tile: TMEM lanes 32 (w % 4) + 16 (w / 4) + [0, 16), read in the
+    // accumulator-fragment layout (16x256b): thread t holds rows t/4 and t/4 + 8, and of every block of 8
+    // columns the two columns 2 (t % 4), 2 (t % 4) + 1.  A row lives in one quad, so its maximum and sum are
+    // two shuffles and no warp waits for another.
+    const int lane_base = (warp & 3) * 32 + (warp >> 2) * 16;
+    const int rA = lane_base + (lane >> 2), rB = rA + 8;   // rows inside the query tile
+    const int cq = 2 * (lane & 3);                         // first of this thread's two columns in a block of 8
+    const uint32_t lane_off = (uint32_t)lane_base << 16;
+    auto quad_max = [](float x) {
+      x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 1));
+      return fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 2));
+    };
+    auto quad_sum = [](float x) {
+      x += __shfl_xor_sync(0xffffffffu, x, 1);
+      return x + __shfl_xor_sync(0xffffffffu, x, 2);
     };
     uint32_t ic = 0, T = 0;
     bool ok = true;
@@ -276,7 +275,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const int q_tok0 = I[0], q_pos0 = I[1], q_rows = I[2], head = I[3], a_len = I[5], b_len = I[7];
       const int split = I[8], n_splits = I[9];
       const int nA = (a_len + 127) >> 7, n = nA + ((b_len + 127) >> 7);
-      float m_used[2] = {0.f, 0.f}, l[2] = {0.f, 0.f};  // l: sum over this thread's columns only
+      // per tile g and row (A, B): running reference maximum and this thread's share of the row sum
+      float mA[2] = {0.f, 0.f}, mB[2] = {0.f, 0.f}, lA[2] = {0.f, 0.f}, lB[2] = {0.f, 0.f};
       for (int j = 0; j < n && ok; ++j, ++T) {
 #pragma unroll
         for (int g = 0; g < 2; ++g) {
@@ -284,119 +284,128 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           ok = mbar_wait(bar_s_full + 8 * g, T & 1, ab, WAIT_FWD_S_FULL);
           if (!ok) break;
           tc_fence_after();
-          // number of leading key columns of this KV tile that the row sees
-          const int limit = (j < nA) ? (a_len - j * 128) : (q_pos0 + g * 128 + r + 1 - (j - nA) * 128);
-          uint32_t s[64];  // raw scores of columns 64 hl .. 64 hl + 63
-          tmem_ld32(tS + hl * 64, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-          tmem_ld32(tS + hl * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+          uint32_t s[64];
+          tmem_ld_16x256b_x16(tS, s);
           tc_wait_ld();
-          if (limit < 128) {
+          // number of leading key columns of this KV tile that rows A and B see
+          const int lim0 = (j < nA) ? (a_len - j * 128) : (q_pos0 + g * 128 + 1 - (j - nA) * 128);
+          const int limA = (j < nA) ? lim0 : lim0 + rA, limB = (j < nA) ? lim0 : lim0 + rB;
+          if (lim0 < 128) {  // same for the whole CTA: a ragged last prompt tile or a tile on the causal diagonal
 #pragma unroll
-            for (int i = 0; i < 64; ++i)
-              if (hl * 64 + i >= limit) s[i] = 0xff800000u;  // -inf: exponentiates to zero
+            for (int i = 0; i < 16; ++i) {
+              const int c = 8 * i + cq;
+              if (c >= limA) s[4 * i] = 0xff800000u;       // -inf: exponentiates to zero
+              if (c + 1 >= limA) s[4 * i + 1] = 0xff800000u;
+              if (c >= limB) s[4 * i + 2] = 0xff800000u;
+              if (c + 1 >= limB) s[4 * i + 3] = 0xff800000u;
+            }
           }
-          // row maximum of the raw scores (the scale is positive, so it commutes with the maximum)
-          float mx0 = -INFINITY, mx1 = -INFINITY;
+          // row maxima of the raw scores (the scale is positive, so it commutes with the maximum)
+          float xA = -INFINITY, xB = -INFINITY;
 #pragma unroll
-          for (int i = 0; i < 64; i += 4) {
-            mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
-            mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+          for (int i = 0; i < 16; ++i) {
+            xA = max3(xA, __uint_as_float(s[4 * i]), __uint_as_float(s[4 * i + 1]));
+            xB = max3(xB, __uint_as_float(s[4 * i + 2]), __uint_as_float(s[4 * i + 3]));
           }
-          mx0 = fmaxf(mx0, mx1);
-          // (the partner has loaded its scores before it gets here, so P may be stored over them below)
-          const float mx = fmaxf(mx0, exchange(mx0, ok)) * p.scale_log2;
-          if (!ok) break;
+          xA = quad_max(xA) * p.scale_log2;
+          xB = quad_max(xB) * p.scale_log2;
           if (j == 0) {
-            m_used[g] = (mx == -INFINITY) ? 0.f : mx;
+            mA[g] = (xA == -INFINITY) ? 0.f : xA;
+            mB[g] = (xB == -INFINITY) ? 0.f : xB;
           } else {
-            const bool need = mx > m_used[g] + kRescaleThreshold;
-            if (__any_sync(0xffffffffu, need)) {  // both warps of the row quadrant see the same rows
+            const bool needA = xA > mA[g] + kRescaleThreshold, needB = xB > mB[g] + kRescaleThreshold;
+            if (__any_sync(0xffffffffu, needA || needB)) {
               ok = mbar_wait(bar_o_full + 8 * g, (T - 1) & 1, ab, WAIT_FWD_O_FULL);  // PV_g(j-1) done
               if (!ok) break;
               tc_fence_after();
-              float alpha = 1.f;
-              if (need) { alpha = ex2(m_used[g] - mx); m_used[g] = mx; l[g] *= alpha; }
+              float alA = 1.f, alB = 1.f;
+              if (needA) { alA = ex2(mA[g] - xA); mA[g] = xA; lA[g] *= alA; }
+              if (needB) { alB = ex2(mB[g] - xB); mB[g] = xB; lB[g] *= alB; }
 #pragma unroll 1
-              for (int c = 0; c < D / 32; ++c) {  // this thread's half of the O row
+              for (int c = 0; c < D / 32; ++c) {
                 uint32_t o[16];
-                tmem_ld16(tO + hl * (D / 2) + c * 16, o);
+                tmem_ld_16x256b_x4(tO + c * 32, o);
                 tc_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                tmem_st16(tO + hl * (D / 2) + c * 16, o);
+                for (int i = 0; i < 4; ++i) {
+                  o[4 * i] = __float_as_uint(__uint_as_float(o[4 * i]) * alA);
+                  o[4 * i + 1] = __float_as_uint(__uint_as_float(o[4 * i + 1]) * alA);
+                  o[4 * i + 2] = __float_as_uint(__uint_as_float(o[4 * i + 2]) * alB);
+                  o[4 * i + 3] = __float_as_uint(__uint_as_float(o[4 * i + 3]) * alB);
+                }
+                tmem_st_16x256b_x4(tO + c * 32, o);
               }
             }
           }
-          // P = exp2(s * scale - m), bf16, stored over the S columns [32 hl + 16 c, +16).  One pair of
+          // P = exp2(s * scale - m), bf16 pairs in the 16x128b layout over the S columns [0, 64).  One block of
           // columns in four takes its exponentials on the FMA pipe, the rest on the special-function unit.
-          float sum0 = 0.f, sum1 = 0.f;
-          const float mg = m_used[g];
+          float sA = 0.f, sB = 0.f;
+          const float ma = mA[g], mb = mB[g];
+          uint32_t pk[32];
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            uint32_t pk[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float x0 = fmaf(__uint_as_float(s[c * 32 + 2 * i]), p.scale_log2, -mg);
-              const float x1 = fmaf(__uint_as_float(s[c * 32 + 2 * i + 1]), p.scale_log2, -mg);
-              float p0, p1;
-              if ((i & 3) == 3) { p0 = ex2_fma(x0); p1 = ex2_fma(x1); }
-              else { p0 = ex2(x0); p1 = ex2(x1); }
-              sum0 += p0;
-              sum1 += p1;
-              pk[i] = pack_bf16(p0, p1);
-            }
-            tmem_st16(tS + hl * 32 + c * 16, pk);
+          for (int i = 0; i < 16; ++i) {
+            const float x0 = fmaf(__uint_as_float(s[4 * i]), p.scale_log2, -ma);
+            const float x1 = fmaf(__uint_as_float(s[4 * i + 1]), p.scale_log2, -ma);
+            const float x2 = fmaf(__uint_as_float(s[4 * i + 2]), p.scale_log2, -mb);
+            const float x3 = fmaf(__uint_as_float(s[4 * i + 3]), p.scale_log2, -mb);
+            float p0, p1, p2, p3;
+            if ((i & 3) == 3) { p0 = ex2_fma(x0); p1 = ex2_fma(x1); p2 = ex2_fma(x2); p3 = ex2_fma(x3); }
+            else { p0 = ex2(x0); p1 = ex2(x1); p2 = ex2(x2); p3 = ex2(x3); }
+            sA += p0 + p1;
+            sB += p2 + p3;
+            pk[2 * i] = pack_bf16(p0, p1);
+            pk[2 * i + 1] = pack_bf16(p2, p3);
           }
-          l[g] += sum0 + sum1;
+          tmem_st_16x128b_x16(tS, pk);
+          lA[g] += sA;
+          lB[g] += sB;
           tc_wait_st();
           tc_fence_before();
           warp_arrive(bar_p_full + 8 * g);
         }
       }
       if (!ok) break;
-      // ---- epilogue: O / l, LSE = ln2 * (m + log2 l); each thread writes its half of the row
+      // ---- epilogue: O / l, LSE = ln2 * (m + log2 l); a thread writes two columns of each block of 8 of its rows
 #pragma unroll
       for (int g = 0; g < 2; ++g) {
         const uint32_t tO = tmem + lane_off + 256 + g * 128;
-        const float lt = l[g] + exchange(l[g], ok);
-        if (!ok) break;
+        const float ltA = quad_sum(lA[g]), ltB = quad_sum(lB[g]);
         ok = mbar_wait(bar_o_full + 8 * g, (T - 1) & 1, ab, WAIT_FWD_O_FULL);
         if (!ok) break;
         tc_fence_after();
-        const float inv_l = 1.f / lt;
-        const long long tok = (long long)q_tok0 + g * 128 + r;
-        const bool valid = g * 128 + r < q_rows;
-        constexpr int HALF = D / 2;
+        const float invA = 1.f / ltA, invB = 1.f / ltB;
+        const long long tokA = (long long)q_tok0 + g * 128 + rA, tokB = tokA + 8;
+        const bool validA = g * 128 + rA < q_rows, validB = g * 128 + rB < q_rows;
 #pragma unroll
-        for (int c = 0; c < HALF / 32; ++c) {
-          uint32_t o[32];
-          tmem_ld32(tO + hl * HALF + c * 32, o);
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[16];
+          tmem_ld_16x256b_x4(tO + c * 32, o);
           tc_wait_ld();
-          if (valid) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int col = c * 32 + 8 * i + cq;
             if (n_splits == 1) {
-              uint4 *dst = reinterpret_cast<uint4 *>(p.o + (tok * p.h_q + head) * D + hl * HALF + c * 32);
-#pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                uint4 w;
-                w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv_l, __uint_as_float(o[8 * v + 1]) * inv_l);
-                w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv_l, __uint_as_float(o[8 * v + 3]) * inv_l);
-                w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv_l, __uint_as_float(o[8 * v + 5]) * inv_l);
-                w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv_l, __uint_as_float(o[8 * v + 7]) * inv_l);
-                dst[v] = w;
-              }
+              if (validA) *reinterpret_cast<uint32_t *>(p.o + (tokA * p.h_q + head) * D + col) =
+                  pack_bf16(__uint_as_float(o[4 * i]) * invA, __uint_as_float(o[4 * i + 1]) * invA);
+              if (validB) *reinterpret_cast<uint32_t *>(p.o + (tokB * p.h_q + head) * D + col) =
+                  pack_bf16(__uint_as_float(o[4 * i + 2]) * invB, __uint_as_float(o[4 * i + 3]) * invB);
             } else {
-              float4 *dst = reinterpret_cast<float4 *>(p.part_o + (((long long)split * p.n_tok + tok) * p.h_q + head) * D + hl * HALF + c * 32);
-#pragma unroll
-              for (int v = 0; v < 8; ++v)
-                dst[v] = make_float4(__uint_as_float(o[4 * v]) * inv_l, __uint_as_float(o[4 * v + 1]) * inv_l,
-                                     __uint_as_float(o[4 * v + 2]) * inv_l, __uint_as_float(o[4 * v + 3]) * inv_l);
+              if (validA) *reinterpret_cast<float2 *>(p.part_o + (((long long)split * p.n_tok + tokA) * p.h_q + head) * D + col) =
+                  make_float2(__uint_as_float(o[4 * i]) * invA, __uint_as_float(o[4 * i + 1]) * invA);
+              if (validB) *reinterpret_cast<float2 *>(p.part_o + (((long long)split * p.n_tok + tokB) * p.h_q + head) * D + col) =
+                  make_float2(__uint_as_float(o[4 * i + 2]) * invB, __uint_as_float(o[4 * i + 3]) * invB);
             }
           }
         }
-        if (valid && hl == 0) {
-          const float lse = (m_used[g] + log2f(lt)) * 0.6931471805599453f;
-          if (n_splits == 1) p.lse[(long long)head * p.n_tok + tok] = lse;
-          else p.part_lse[((long long)split * p.h_q + head) * p.n_tok + tok] = lse;
+        if ((lane & 3) == 0) {
+          const float lseA = (mA[g] + log2f(ltA)) * 0.6931471805599453f, lseB = (mB[g] + log2f(ltB)) * 0.6931471805599453f;
+          if (n_splits == 1) {
+            if (validA) p.lse[(long long)head * p.n_tok + tokA] = lseA;
+            if (validB) p.lse[(long long)head * p.n_tok + tokB] = lseB;
+          } else {
+            if (validA) p.part_lse[((long long)split * p.h_q + head) * p.n_tok + tokA] = lseA;
+            if (validB) p.part_lse[((long long)split * p.h_q + head) * p.n_tok + tokB] = lseB;
+          }
         }
         tc_fence_before();
         warp_arrive(bar_o_empty + 8 * g);
