@@ -146,3 +146,81 @@ def brute_force_makespan(weights, n_lanes):
             loads[l] -= weights[i]
     rec(0)
     return best[0]
+
+
+# --------------------------------------------------------------------------- #
+# Replay-grid assignment (Sec. 3.4 "Replay units and grid assignment", Eq. 6).
+#
+# Units k = 0..U-1 with work w_k are placed on a grid of b rounds x s lanes,
+# X_k = (round, lane).  Lanes of a round run concurrently and rounds run one
+# after the other, so the predicted critical path is
+#     sum over rounds of ( max over lanes of ( sum of w_k placed there ) ).
+# The paper adds per-lane memory limits; here a unit also has a size m_k and a
+# (round, lane) cell holds at most `cap` of it (cap None: no limit).  Without a
+# limit one round is always enough, because merging rounds never lengthens the
+# path; the limit is what makes several rounds necessary.
+#
+# grid_objective is Eq. 6 written out; brute_force_grid is its definition as a
+# minimum over every assignment (tiny inputs only); greedy_grid restates the
+# largest-first rule the library uses above the exact-solver cap, tie-breaks
+# included, for a bit-exact comparison.  Test infrastructure only.
+
+
+def grid_objective(weights, rounds, lanes, n_rounds, n_lanes):
+    load = np.zeros((n_rounds, n_lanes), dtype=np.int64)
+    for w, t, j in zip(weights, rounds, lanes):
+        load[t, j] += int(w)
+    return int(load.max(axis=1).sum())
+
+
+def grid_feasible(mem, rounds, lanes, n_rounds, n_lanes, cap):
+    if cap is None:
+        return True
+    used = np.zeros((n_rounds, n_lanes), dtype=np.int64)
+    for m, t, j in zip(mem, rounds, lanes):
+        used[t, j] += int(m)
+    return bool((used <= cap).all())
+
+
+def brute_force_grid(weights, mem, n_rounds, n_lanes, cap):
+    """Minimum of Eq. 6 over all (n_rounds * n_lanes)^U assignments; None if no assignment fits the limit."""
+    import itertools
+    cells = [(t, j) for t in range(n_rounds) for j in range(n_lanes)]
+    best = None
+    for choice in itertools.product(range(len(cells)), repeat=len(weights)):
+        rounds = [cells[c][0] for c in choice]
+        lanes = [cells[c][1] for c in choice]
+        if not grid_feasible(mem, rounds, lanes, n_rounds, n_lanes, cap):
+            continue
+        v = grid_objective(weights, rounds, lanes, n_rounds, n_lanes)
+        if best is None or v < best:
+            best = v
+    return best
+
+
+def greedy_grid(weights, mem, n_rounds, n_lanes, cap):
+    """Largest-first greedy: units by weight descending (index ascending on ties); each goes to the cell that
+    fits and gives the smallest critical path afterwards, then the smallest cell load, then the lowest round,
+    then the lowest lane.  Returns (rounds, lanes, objective) or None if some unit fits nowhere."""
+    U = len(weights)
+    load = [[0] * n_lanes for _ in range(n_rounds)]
+    used = [[0] * n_lanes for _ in range(n_rounds)]
+    rounds, lanes = [0] * U, [0] * U
+    for k in sorted(range(U), key=lambda i: (-int(weights[i]), i)):
+        best = None
+        for t in range(n_rounds):
+            peak = max(load[t])
+            for j in range(n_lanes):
+                if cap is not None and used[t][j] + int(mem[k]) > cap:
+                    continue
+                new = load[t][j] + int(weights[k])
+                key = (max(peak, new) - peak, new, t, j)  # growth of this round's maximum = growth of the path
+                if best is None or key < best[0]:
+                    best = (key, t, j)
+        if best is None:
+            return None
+        _, t, j = best
+        load[t][j] += int(weights[k])
+        used[t][j] += int(mem[k])
+        rounds[k], lanes[k] = t, j
+    return rounds, lanes, sum(max(r) for r in load)

@@ -230,3 +230,50 @@ def test_redundancy_fraction():
     for P, G, R, want in [(256, 4, 128, 1.501), (8192, 8, 2048, 2.273), (65536, 8, 1024, 6.591)]:
         pre, rep, flat = ora.valid_pairs(ora.TreeBatch([P], [[R] * G], 1, 1, 8))
         assert abs(flat / (pre + rep) - want) < 1e-3
+
+
+# --------------------------------------------------------------------------- #
+# Replay-grid assignment (Eq. 6): pins of the brute-force definition
+def test_grid_assignment_definition_reduces_to_known_cases():
+    from oracle import packing as pk
+    rng = np.random.default_rng(11)
+    for _ in range(12):
+        U = int(rng.integers(1, 7))
+        w = [int(x) for x in rng.integers(1, 40, size=U)]
+        m = [1] * U
+        # one lane: every round's maximum is its sum, so any assignment costs the total work
+        assert pk.brute_force_grid(w, m, 2, 1, None) == sum(w)
+        # no memory limit: merging rounds never lengthens the path, so several rounds buy nothing and the
+        # optimum is the classical makespan on s machines (an independent exhaustive routine)
+        for s in (2, 3):
+            assert pk.brute_force_grid(w, m, 2, s, None) == pk.brute_force_makespan(w, s)
+            assert pk.brute_force_grid(w, m, 1, s, None) == pk.brute_force_makespan(w, s)
+        # at least as many cells in one round as units: the longest unit alone
+        assert pk.brute_force_grid(w, m, 1, U, None) == max(w)
+    # a hand-worked case with a limit of one unit per cell: 2 rounds x 2 lanes, works 5, 4, 3, 1
+    # -> rounds {5,4} and {3,1} cost 5 + 3 = 8; {5,1},{4,3} costs 5 + 4 = 9; {5,3},{4,1} costs 5 + 4 = 9
+    assert pk.brute_force_grid([5, 4, 3, 1], [1, 1, 1, 1], 2, 2, 1) == 8
+    # five units do not fit four cells of one unit each
+    assert pk.brute_force_grid([1, 1, 1, 1, 1], [1] * 5, 2, 2, 1) is None
+    # a tighter limit can only lengthen the path
+    w, m = [9, 7, 6, 5, 4, 2], [3, 2, 2, 1, 1, 1]
+    vals = [pk.brute_force_grid(w, m, 2, 2, cap) for cap in (3, 4, 5, 10)]
+    assert all(a >= b for a, b in zip(vals, vals[1:])) and vals[-1] == pk.brute_force_makespan(w, 2)
+
+
+def test_grid_greedy_is_valid_and_never_beats_the_optimum():
+    from oracle import packing as pk
+    rng = np.random.default_rng(12)
+    for _ in range(30):
+        U = int(rng.integers(1, 7))
+        w = [int(x) for x in rng.integers(1, 30, size=U)]
+        m = [int(x) for x in rng.integers(1, 4, size=U)]
+        b, s = int(rng.integers(1, 3)), int(rng.integers(1, 3))
+        cap = None if rng.random() < 0.4 else int(rng.integers(3, 8))
+        opt = pk.brute_force_grid(w, m, b, s, cap)
+        g = pk.greedy_grid(w, m, b, s, cap)
+        if g is None:
+            continue  # greedy may fail to pack what an exhaustive search can
+        rounds, lanes, val = g
+        assert opt is not None and pk.grid_feasible(m, rounds, lanes, b, s, cap)
+        assert val == pk.grid_objective(w, rounds, lanes, b, s) >= opt
