@@ -250,6 +250,26 @@ int augtree_get_kernel_time(const augtree_plan_t *plan, int kernel, float *total
 /* Number of kernel launches the library has enqueued since it was loaded. */
 long long augtree_launch_count(void);
 
+/*
+ * Replay-grid assignment (Sec. 3.4 "Replay units and grid assignment", Eq. 6; the AssignGrid step of
+ * Algorithm 1).  Host only, no device work.  n_units replay units with work weight[k] >= 0 and size
+ * size[k] >= 0 are placed on a grid of n_rounds x n_lanes cells, unit k into cell (round_out[k],
+ * lane_out[k]).  Lanes of a round run concurrently and rounds run in sequence, so the predicted
+ * critical path is  sum over rounds of (max over lanes of (sum of the weights placed there)),  which
+ * is what is minimised and returned in *critical_path; a cell holds at most cell_cap of size
+ * (cell_cap <= 0: no limit, size may then be NULL).  Up to exact_max_units units (0 selects 12, at
+ * most 16) the minimum is exact (dynamic programming over subsets) and *solved_exactly is 1; above
+ * it units are placed largest first (ties: lower index), each into the cell that fits and lengthens
+ * the path least, then the lightest such cell, then the lowest round, then the lowest lane, and
+ * *solved_exactly is 0.  All arrays are host memory owned by the caller; critical_path and
+ * solved_exactly may be NULL.  Returns AUGTREE_ERR_INVALID_ARG for bad arguments and
+ * AUGTREE_ERR_UNSUPPORTED when the units cannot be packed under cell_cap (exact solver: no packing
+ * exists; greedy: none was found) or the grid is larger than 1024 rounds x 65536 lanes.
+ */
+int augtree_assign_grid(const int64_t *weight, const int64_t *size, int n_units, int n_rounds, int n_lanes,
+                        int64_t cell_cap, int exact_max_units, int32_t *round_out, int32_t *lane_out,
+                        int64_t *critical_path, int32_t *solved_exactly);
+
 const char *augtree_status_string(int status);
 
 #ifdef __cplusplus

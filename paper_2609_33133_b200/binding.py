@@ -31,7 +31,7 @@ FWD_ITEM_INTS, BWD_ITEM_INTS = 12, 8
 EXPORTS = ["augtree_plan_create", "augtree_plan_destroy", "augtree_plan_workspace_bytes", "augtree_plan_metadata",
            "augtree_prefill_fwd", "augtree_replay_fwd", "augtree_replay_bwd", "augtree_prefill_bwd",
            "augtree_last_device_status", "augtree_launch_count", "augtree_status_string",
-           "augtree_set_timing", "augtree_get_kernel_time", "augtree_replay_fwd_static"]
+           "augtree_set_timing", "augtree_get_kernel_time", "augtree_replay_fwd_static", "augtree_assign_grid"]
 
 
 class Desc(C.Structure):
@@ -60,6 +60,10 @@ lib.augtree_status_string.restype = C.c_char_p
 lib.augtree_status_string.argtypes = [C.c_int]
 
 
+_i64p, _i32p = C.POINTER(C.c_int64), C.POINTER(C.c_int32)
+lib.augtree_assign_grid.argtypes = [_i64p, _i64p, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int, _i32p, _i32p, _i64p, _i32p]
+
+
 class AugtreeError(RuntimeError):
     def __init__(self, code, where):
         self.code = code
@@ -73,6 +77,18 @@ def _check(code, where):
 
 def _ptr(t):
     return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def assign_grid(weight, size=None, n_rounds=1, n_lanes=1, cell_cap=0, exact_max_units=0):
+    """augtree_assign_grid: returns (round[k], lane[k], critical path, solved exactly)."""
+    n = len(weight)
+    w = (C.c_int64 * max(n, 1))(*[int(x) for x in weight])
+    m = None if size is None else (C.c_int64 * max(n, 1))(*[int(x) for x in size])
+    rounds, lanes = (C.c_int32 * max(n, 1))(), (C.c_int32 * max(n, 1))()
+    path, exact = C.c_int64(0), C.c_int32(0)
+    _check(lib.augtree_assign_grid(w, m, n, n_rounds, n_lanes, int(cell_cap), exact_max_units, rounds, lanes,
+                                   C.byref(path), C.byref(exact)), "augtree_assign_grid")
+    return list(rounds[:n]), list(lanes[:n]), int(path.value), bool(exact.value)
 
 
 def launch_count() -> int:

@@ -1,0 +1,152 @@
+// Replay-grid assignment (Sec. 3.4 "Replay units and grid assignment", Eq. 6): host only.
+//
+// U units with work w_k and size m_k go onto a grid of b rounds x s lanes.  Lanes of a round
+// run side by side and rounds one after the other, so the predicted critical path is the sum
+// over rounds of the heaviest lane of the round; a (round, lane) cell holds at most `cap` of
+// size.  Up to `exact_max_units` units the minimum is found exactly by dynamic programming
+// over subsets (the paper's bounded AssignGrid); above it units are placed largest first.
+#include <algorithm>
+#include <cstdint>
+#include <limits>
+#include <numeric>
+#include <vector>
+
+#include "../../include/augtree.h"
+
+namespace {
+
+constexpr int64_t kInf = std::numeric_limits<int64_t>::max() / 4;
+constexpr int kHardMaxExact = 16;  // 3^16 subset pairs is the most the exact solver is allowed
+
+// Exact solver.  lane_best[j][S]: least possible heaviest lane when the units of S share j lanes
+// of one round (kInf if they do not fit); round_best[t][S]: least path when S is spread over t rounds.
+// Both recurrences peel off the part that contains the lowest unit of S, which visits every
+// partition once.
+struct ExactGrid {
+  int U, b, s;
+  std::vector<int64_t> wsum, msum;
+  std::vector<std::vector<int64_t>> lane_best, round_best;
+  std::vector<std::vector<uint32_t>> lane_pick, round_pick;
+
+  bool solve(const int64_t *w, const int64_t *m, int64_t cap) {
+    const uint32_t full = (1u << U) - 1;
+    wsum.assign(full + 1, 0);
+    msum.assign(full + 1, 0);
+    for (uint32_t S = 1; S <= full; ++S) {
+      const int k = __builtin_ctz(S);
+      wsum[S] = wsum[S & (S - 1)] + w[k];
+      msum[S] = msum[S & (S - 1)] + (m ? m[k] : 0);
+    }
+    auto fits = [&](uint32_t T) { return cap <= 0 || msum[T] <= cap; };
+    lane_best.assign(s + 1, std::vector<int64_t>(full + 1, kInf));
+    lane_pick.assign(s + 1, std::vector<uint32_t>(full + 1, 0));
+    for (int j = 0; j <= s; ++j) lane_best[j][0] = 0;
+    for (int j = 1; j <= s; ++j)
+      for (uint32_t S = 1; S <= full; ++S) {
+        const uint32_t low = S & (~S + 1), rest = S ^ low;
+        // T = low | (any subset of rest): the lane that takes the lowest unit
+        for (uint32_t sub = rest;; sub = (sub - 1) & rest) {
+          const uint32_t T = sub | low;
+          if (fits(T) && lane_best[j - 1][S ^ T] < kInf) {
+            const int64_t v = std::max(wsum[T], lane_best[j - 1][S ^ T]);
+            if (v < lane_best[j][S]) { lane_best[j][S] = v; lane_pick[j][S] = T; }
+          }
+          if (sub == 0) break;
+        }
+      }
+    round_best.assign(b + 1, std::vector<int64_t>(full + 1, kInf));
+    round_pick.assign(b + 1, std::vector<uint32_t>(full + 1, 0));
+    for (int t = 0; t <= b; ++t) round_best[t][0] = 0;
+    for (int t = 1; t <= b; ++t)
+      for (uint32_t S = 1; S <= full; ++S) {
+        const uint32_t low = S & (~S + 1), rest = S ^ low;
+        for (uint32_t sub = rest;; sub = (sub - 1) & rest) {
+          const uint32_t T = sub | low;
+          if (lane_best[s][T] < kInf && round_best[t - 1][S ^ T] < kInf) {
+            const int64_t v = lane_best[s][T] + round_best[t - 1][S ^ T];
+            if (v < round_best[t][S]) { round_best[t][S] = v; round_pick[t][S] = T; }
+          }
+          if (sub == 0) break;
+        }
+      }
+    return round_best[b][full] < kInf;
+  }
+
+  void unpack(int32_t *round_out, int32_t *lane_out) const {
+    uint32_t S = (1u << U) - 1;
+    int t = b, round = 0;
+    while (S) {
+      const uint32_t R = round_pick[t][S];
+      uint32_t L = R;
+      int j = s, lane = 0;
+      while (L) {
+        const uint32_t T = lane_pick[j][L];
+        for (uint32_t x = T; x; x &= x - 1) {
+          const int k = __builtin_ctz(x);
+          round_out[k] = round;
+          lane_out[k] = lane;
+        }
+        L ^= T; --j; ++lane;
+      }
+      S ^= R; --t; ++round;
+    }
+  }
+};
+
+}  // namespace
+
+extern "C" int augtree_assign_grid(const int64_t *weight, const int64_t *size, int n_units, int n_rounds, int n_lanes,
+                                   int64_t cell_cap, int exact_max_units, int32_t *round_out, int32_t *lane_out,
+                                   int64_t *critical_path, int32_t *solved_exactly) {
+  if (n_units < 0 || n_rounds < 1 || n_lanes < 1 || (n_units > 0 && (!weight || !round_out || !lane_out))) return AUGTREE_ERR_INVALID_ARG;
+  if (cell_cap > 0 && !size && n_units > 0) return AUGTREE_ERR_INVALID_ARG;
+  if (n_rounds > 1024 || n_lanes > 65536) return AUGTREE_ERR_UNSUPPORTED;
+  for (int k = 0; k < n_units; ++k)
+    if (weight[k] < 0 || (size && size[k] < 0) || weight[k] > kInf / (n_units + 1)) return AUGTREE_ERR_INVALID_ARG;
+  if (exact_max_units <= 0) exact_max_units = 12;
+  exact_max_units = std::min(exact_max_units, kHardMaxExact);
+  int64_t path = 0;
+  bool exact = false;
+  if (n_units == 0) {
+    exact = true;
+  } else if (n_units <= exact_max_units) {
+    ExactGrid g;
+    g.U = n_units; g.b = n_rounds; g.s = n_lanes;
+    // more lanes (rounds) than units cannot help: cap them so that the tables stay small
+    g.s = std::min(g.s, n_units);
+    g.b = std::min(g.b, n_units);
+    if (!g.solve(weight, size, cell_cap)) return AUGTREE_ERR_UNSUPPORTED;  // the units do not fit the grid
+    g.unpack(round_out, lane_out);
+    path = g.round_best[g.b][(1u << n_units) - 1];
+    exact = true;
+  } else {
+    // largest first; each unit to the cell that fits and lengthens the path least, then to the lightest
+    // such cell, then the lowest round, then the lowest lane
+    std::vector<int32_t> ids(n_units);
+    std::iota(ids.begin(), ids.end(), 0);
+    std::stable_sort(ids.begin(), ids.end(), [&](int32_t a, int32_t c) { return weight[a] > weight[c]; });
+    std::vector<int64_t> load((size_t)n_rounds * n_lanes, 0), used((size_t)n_rounds * n_lanes, 0), peak(n_rounds, 0);
+    for (int32_t k : ids) {
+      int bt = -1, bj = -1;
+      int64_t b_grow = 0, b_new = 0;
+      for (int t = 0; t < n_rounds; ++t)
+        for (int j = 0; j < n_lanes; ++j) {
+          const size_t c = (size_t)t * n_lanes + j;
+          if (cell_cap > 0 && used[c] + size[k] > cell_cap) continue;
+          const int64_t nw = load[c] + weight[k], grow = std::max(peak[t], nw) - peak[t];
+          if (bt < 0 || grow < b_grow || (grow == b_grow && nw < b_new)) { bt = t; bj = j; b_grow = grow; b_new = nw; }
+        }
+      if (bt < 0) return AUGTREE_ERR_UNSUPPORTED;
+      const size_t c = (size_t)bt * n_lanes + bj;
+      load[c] += weight[k];
+      if (size) used[c] += size[k];
+      peak[bt] = std::max(peak[bt], load[c]);
+      round_out[k] = bt;
+      lane_out[k] = bj;
+    }
+    for (int t = 0; t < n_rounds; ++t) path += peak[t];
+  }
+  if (critical_path) *critical_path = path;
+  if (solved_exactly) *solved_exactly = exact ? 1 : 0;
+  return AUGTREE_OK;
+}

@@ -128,3 +128,70 @@ def test_greedy_assignment_within_lpt_bound():
         got = packing.makespan(w, ptr, order)
         opt = packing.brute_force_makespan(w, m)
         assert opt <= got <= opt * (4 / 3 - 1 / (3 * m)) + 1e-9
+
+
+# --------------------------------------------------------------------------- #
+# Replay-grid assignment (Eq. 6) against the oracle's brute-force definition
+def test_assign_grid_exact_matches_brute_force(binding):
+    from oracle import packing as pk
+    rng = np.random.default_rng(21)
+    for trial in range(60):
+        U = int(rng.integers(1, 8))
+        w = [int(x) for x in rng.integers(0, 50, size=U)]
+        m = [int(x) for x in rng.integers(1, 5, size=U)]
+        b, s = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        if (b * s) ** U > 300000:
+            b = 1
+        cap = None if trial % 3 == 0 else int(rng.integers(2, 9))
+        want = pk.brute_force_grid(w, m, b, s, cap)
+        if want is None:
+            with pytest.raises(binding.AugtreeError) as e:
+                binding.assign_grid(w, m, b, s, cell_cap=cap or 0)
+            assert e.value.code == -2  # unsupported: no packing exists
+            continue
+        rounds, lanes, path, exact = binding.assign_grid(w, m, b, s, cell_cap=cap or 0)
+        # the optimal value is unique; the assignment need only be valid and reach it
+        assert exact and path == want
+        assert all(0 <= t < b for t in rounds) and all(0 <= j < s for j in lanes)
+        assert pk.grid_feasible(m, rounds, lanes, b, s, cap)
+        assert pk.grid_objective(w, rounds, lanes, b, s) == want
+
+
+def test_assign_grid_greedy_is_bit_exact_and_bounded(binding):
+    from oracle import packing as pk
+    rng = np.random.default_rng(22)
+    for trial in range(40):
+        U = int(rng.integers(1, 40))
+        w = [int(x) for x in rng.integers(1, 1000, size=U)]
+        m = [int(x) for x in rng.integers(1, 9, size=U)]
+        b, s = int(rng.integers(1, 4)), int(rng.integers(1, 6))
+        cap = None if trial % 2 == 0 else int(rng.integers(8, 40))
+        want = pk.greedy_grid(w, m, b, s, cap)
+        if U == 1:
+            continue  # a single unit always takes the exact path
+        if want is None:
+            with pytest.raises(binding.AugtreeError):
+                binding.assign_grid(w, m, b, s, cell_cap=cap or 0, exact_max_units=1)
+            continue
+        rounds, lanes, path, exact = binding.assign_grid(w, m, b, s, cell_cap=cap or 0, exact_max_units=1)
+        assert not exact and (rounds, lanes, path) == (want[0], want[1], want[2])
+        if U <= 12:  # the exact solver can only be better
+            _, _, opt, ex = binding.assign_grid(w, m, b, s, cell_cap=cap or 0)
+            assert ex and opt <= path
+    # sixteen units, exact: the classical bound for one round, and a larger instance still answers quickly
+    w = [int(x) for x in np.random.default_rng(23).integers(1, 100, size=14)]
+    _, _, opt, ex = binding.assign_grid(w, None, 1, 4, exact_max_units=16)
+    assert ex and max(max(w), -(-sum(w) // 4)) <= opt <= pk.makespan(w, *pk.assign_lanes(w, 4))
+
+
+def test_assign_grid_rejects_bad_arguments(binding):
+    with pytest.raises(binding.AugtreeError) as e:
+        binding.assign_grid([1, 2], None, 0, 1)
+    assert e.value.code == -1
+    with pytest.raises(binding.AugtreeError) as e:
+        binding.assign_grid([1, -2], None, 1, 1)
+    assert e.value.code == -1
+    with pytest.raises(binding.AugtreeError) as e:
+        binding.assign_grid([1, 2], None, 1, 1, cell_cap=3)  # a limit needs sizes
+    assert e.value.code == -1
+    assert binding.assign_grid([], None, 2, 2) == ([], [], 0, True)
