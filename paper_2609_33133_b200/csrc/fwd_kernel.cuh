@@ -144,7 +144,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const uint32_t q_lo0 = sdesc_lo(sQ, 16), q_lo1 = sdesc_lo(sQ + TILE, 16);
       // a look that succeeded makes the wait unnecessary (every lane sees the same barrier state)
       auto need = [&](bool have, uint32_t bar, uint32_t par, int site) -> bool {
-        if (!have && !mbar_spin(bar, par, ab, site)) return false;
+        if (!have && !mbar_wait(bar, par, ab, site)) return false;
         tc_fence_after();
         return true;
       };

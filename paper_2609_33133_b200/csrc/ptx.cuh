@@ -85,25 +85,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
   }
 }
 
-// The same wait as a pure spin on test_wait: for hand-offs on the critical path, where the time try_wait
-// takes to resume a suspended warp would be paid on every tile.
-__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity, const AbortCtx &ab, int site) {
-  if (mbar_test(bar, parity)) return true;
-  const long long t0 = clock64();
-  unsigned spins = 0;
-  while (true) {
-    if (mbar_test(bar, parity)) return true;
-    if ((++spins & 1023u) == 0) {
-      if (*ab.flag) return false;
-      if (clock64() - t0 > kWaitBudgetClocks) {
-        *ab.flag = 1;
-        if (atomicCAS(ab.status, 0, -5) == 0) ab.status[1] = site;
-        return false;
-      }
-    }
-  }
-}
-
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
