@@ -31,6 +31,7 @@ SMALL = [
     _wl("prompt-only", [200, 130], [[], []], 2, 1, 128, 14),
     _wl("tiny", [1], [[1]], 1, 1, 64, 15),
     _wl("g7", [640], [[192] * 3], 14, 2, 128, 16),
+    _wl("d64-multi", [900, 260], [[700, 300, 129], [515]], 8, 2, 64, 17),   # head dim 64 over many tiles, GQA 4:1
 ]
 
 
@@ -55,6 +56,14 @@ def test_split_prompt_kv_matches_oracle(B, splits):
     w = _wl("split", [1100, 200], [[130, 64], [257]], 4, 2, 128, 21)
     t = wl.make_tensors(w)
     got, plan = pu.run_gpu(B, w, t, kv_splits=splits)
+    assert plan.metadata(B.TBL_GROUP_SPLITS).max() > 1
+    pu.assert_parity(got, pu.run_oracle(w, t))
+
+
+def test_split_prompt_kv_head_dim_64(B):
+    w = _wl("split-d64", [1300], [[200, 333]], 4, 1, 64, 22)
+    t = wl.make_tensors(w)
+    got, plan = pu.run_gpu(B, w, t, kv_splits=4)
     assert plan.metadata(B.TBL_GROUP_SPLITS).max() > 1
     pu.assert_parity(got, pu.run_oracle(w, t))
 
