@@ -14,9 +14,9 @@
 //   dV  += P^T dO      (A = P^T from TMEM)
 //   dK  += dS^T Q      (A = dS^T from TMEM)
 //
-// Warp roles (320 threads): warps 0-7 element-wise (warp w: TMEM lanes
-// 32*(w%4).., query columns 64*(w/4)..), warp 8 lane 0 TMA loads, warp 9 lane 0
-// MMA issue.  TMEM columns: R0 [0,128) S^T, overwritten in place by P^T (bf16);
+// Warp roles (576 threads): warps 0-15 element-wise (warp w: TMEM lanes
+// 32*(w%4).., query columns 32*(w/4)..), warp 16 lane 0 TMA loads, warp 17 MMA
+// issue (whole warp in lockstep, one elected lane).  TMEM columns: R0 [0,128) S^T, overwritten in place by P^T (bf16);
 // R1 [128,256) dP^T, overwritten in place by dS^T (bf16); dV at 256; dK at 256 + D.
 // MMA issue order in steady state: dP(T), dV(T), S(T+1), dK(T); the tensor pipe
 // executes in order, so S(T+1) may overwrite R0 once dV(T) is issued and
@@ -42,7 +42,7 @@ struct BwdParams {
   int *status;
 };
 
-constexpr int kBwdThreads = 320;
+constexpr int kBwdThreads = 576;  // 16 element-wise warps, TMA warp, MMA warp
 
 template <int D>
 struct BwdSmem {
@@ -95,12 +95,12 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       mbar_init(bar_q_full + 8 * s, 1); mbar_init(bar_q_empty + 8 * s, 1);
       mbar_init(bar_do_full + 8 * s, 1); mbar_init(bar_do_empty + 8 * s, 1);
     }
-    mbar_init(bar_s_full, 1); mbar_init(bar_p_ready, 8); mbar_init(bar_dp_full, 1); mbar_init(bar_ds_ready, 8);
-    mbar_init(bar_acc_full, 1); mbar_init(bar_acc_empty, 8);
+    mbar_init(bar_s_full, 1); mbar_init(bar_p_ready, 16); mbar_init(bar_dp_full, 1); mbar_init(bar_ds_ready, 16);
+    mbar_init(bar_acc_full, 1); mbar_init(bar_acc_empty, 16);
     *abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == 9) { tmem_alloc(smem_u32((const void *)tmem_slot), 512); tmem_relinquish(); }
+  if (warp == 17) { tmem_alloc(smem_u32((const void *)tmem_slot), 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -110,7 +110,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   const int rep = p.h_q / p.h_kv;
   const int it_begin = p.lane_ptr[blockIdx.x], it_end = p.lane_ptr[blockIdx.x + 1];
 
-  if (warp == 8) {
+  if (warp == 16) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_do); tma_prefetch_desc(&tm_k0);
@@ -150,7 +150,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == 17) {
     // -------------------------------------------------------------- MMA issuer
     // The whole warp runs the loops in lockstep and one elected lane issues (warp-uniform descriptor
     // arithmetic: few instructions per MMA, which matters next to two busy element-wise warps on the same
@@ -214,10 +214,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           }
           ok = need(have_p, bar_p_ready, T & 1, WAIT_BWD_PDS_FULL);
           if (!ok) break;
-          // (query columns 16k..16k+15: P^T sits at R0 columns 8k (k<4) or 64+8(k-4))
+          // (query columns 16k..16k+15: P^T sits at R0 columns 32 (k / 2) + 8 (k % 2), over its own thread's S^T)
           mma_group<8>(elected,
                        [&](int k) {
-                         mma_ts2(tDV, tR0 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), dom_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
+                         mma_ts2(tDV, tR0 + 32 * (k >> 1) + 8 * (k & 1), dom_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
                        },
                        [&]() { have_q = more && mbar_test(bar_q_full + 8 * st1, par1); });
           if (elected) tc_commit(bar_do_empty + 8 * st);
@@ -236,7 +236,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           have_do = false;
           mma_group<8>(elected,
                        [&](int k) {
-                         mma_ts2(tDK, tR1 + (k < 4 ? k * 8 : 64 + (k - 4) * 8), qm_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
+                         mma_ts2(tDK, tR1 + 32 * (k >> 1) + 8 * (k & 1), qm_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
                        },
                        [&]() { have_do = more && mbar_test(bar_do_full + 8 * st1, par1); });
           if (elected) tc_commit(bar_q_empty + 8 * st);
@@ -246,13 +246,16 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       }
     }
   } else {
-    // ------------------------------------------------------- element-wise warps 0-7
+    // ------------------------------------------------------- element-wise warps 0-15
+    // Warp w: TMEM lanes (key rows) 32 (w % 4) .., query columns 32 (w / 4) .. of every tile: four threads per
+    // key row.  The phases are bound by the latency of their loads and special-function results, which four
+    // warps per scheduler hide better than two.
     const int lg = warp & 3, ch = warp >> 2;
     const int r = lg * 32 + lane;  // TMEM lane = key row
     const uint32_t lane_off = (uint32_t)(lg * 32) << 16;
     uint32_t ic = 0, T = 0;
     bool ok = true;
-    float pr[64];  // P^T of the current pair: key r, query columns 64*ch .. 64*ch+63
+    float pr[32];  // P^T of the current pair: key r, query columns 32*ch .. 32*ch+31
 
     // P^T(Tn) from S^T(Tn): wait, load, exponentiate, store bf16 over S^T, signal
     auto make_p = [&](uint32_t Tn, int q_base, int kv_pos0, int mode, bool key_valid) -> bool {
@@ -260,16 +263,15 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       if (!mbar_wait(bar_q_full + 8 * st, (Tn / NST) & 1, ab, WAIT_BWD_QDO_FULL)) return false;  // row statistics landed
       if (!mbar_wait(bar_s_full, Tn & 1, ab, WAIT_BWD_S_FULL)) return false;
       tc_fence_after();
-      const float *lse2 = reinterpret_cast<const float *>(smem_raw + SM::kOffStats + st * 1024) + ch * 64;
+      const float *lse2 = reinterpret_cast<const float *>(smem_raw + SM::kOffStats + st * 1024) + ch * 32;
       // query column (inside the tile) from which this key is visible
       const int lo = mode ? 0 : (kv_pos0 + r - q_base);
-      const bool all_visible = key_valid && lo <= ch * 64;
-      uint32_t sv[64];
-      tmem_ld32(tR0 + lane_off + ch * 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
-      tmem_ld32(tR0 + lane_off + ch * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+      const bool all_visible = key_valid && lo <= ch * 32;
+      uint32_t sv[32];
+      tmem_ld32(tR0 + lane_off + ch * 32, sv);
       tc_wait_ld();
 #pragma unroll
-      for (int i = 0; i < 64; i += 4) {
+      for (int i = 0; i < 32; i += 4) {
         const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + i);
         pr[i + 0] = ex2(fmaf(__uint_as_float(sv[i + 0]), p.scale_log2, -l4.x));
         pr[i + 1] = ex2(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -l4.y));
@@ -278,15 +280,14 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       }
       if (!all_visible) {
 #pragma unroll
-        for (int i = 0; i < 64; ++i)
-          if (!key_valid || ch * 64 + i < lo) pr[i] = 0.f;
+        for (int i = 0; i < 32; ++i)
+          if (!key_valid || ch * 32 + i < lo) pr[i] = 0.f;
       }
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      {
         uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(pr[c * 32 + 2 * i], pr[c * 32 + 2 * i + 1]);
-        tmem_st16(tR0 + lane_off + ch * 64 + c * 16, pk);
+        for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(pr[2 * i], pr[2 * i + 1]);
+        tmem_st16(tR0 + lane_off + ch * 32, pk);
       }
       tc_wait_st();
       tc_fence_before();
@@ -316,26 +317,22 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             if (!ok) break;
             tc_fence_after();
             {
-              const float *dl = reinterpret_cast<const float *>(smem_raw + SM::kOffStats + st * 1024) + 128 + ch * 64;
-              uint32_t dpv[64];
-              tmem_ld32(tR1 + lane_off + ch * 64, *reinterpret_cast<uint32_t(*)[32]>(&dpv[0]));
-              tmem_ld32(tR1 + lane_off + ch * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&dpv[32]));
+              const float *dl = reinterpret_cast<const float *>(smem_raw + SM::kOffStats + st * 1024) + 128 + ch * 32;
+              uint32_t dpv[32];
+              tmem_ld32(tR1 + lane_off + ch * 32, dpv);
               tc_wait_ld();
+              uint32_t dd[16];
 #pragma unroll
-              for (int c = 0; c < 2; ++c) {
-                uint32_t dd[16];
-#pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                  const float4 d4 = *reinterpret_cast<const float4 *>(dl + c * 32 + i);
-                  const float a0 = pr[c * 32 + i + 0] * fmaf(__uint_as_float(dpv[c * 32 + i + 0]), p.scale, -d4.x);
-                  const float a1 = pr[c * 32 + i + 1] * fmaf(__uint_as_float(dpv[c * 32 + i + 1]), p.scale, -d4.y);
-                  const float a2 = pr[c * 32 + i + 2] * fmaf(__uint_as_float(dpv[c * 32 + i + 2]), p.scale, -d4.z);
-                  const float a3 = pr[c * 32 + i + 3] * fmaf(__uint_as_float(dpv[c * 32 + i + 3]), p.scale, -d4.w);
-                  dd[i / 2] = pack_bf16(a0, a1);
-                  dd[i / 2 + 1] = pack_bf16(a2, a3);
-                }
-                tmem_st16(tR1 + lane_off + ch * 64 + c * 16, dd);
+              for (int i = 0; i < 32; i += 4) {
+                const float4 d4 = *reinterpret_cast<const float4 *>(dl + i);
+                const float a0 = pr[i + 0] * fmaf(__uint_as_float(dpv[i + 0]), p.scale, -d4.x);
+                const float a1 = pr[i + 1] * fmaf(__uint_as_float(dpv[i + 1]), p.scale, -d4.y);
+                const float a2 = pr[i + 2] * fmaf(__uint_as_float(dpv[i + 2]), p.scale, -d4.z);
+                const float a3 = pr[i + 3] * fmaf(__uint_as_float(dpv[i + 3]), p.scale, -d4.w);
+                dd[i / 2] = pack_bf16(a0, a1);
+                dd[i / 2 + 1] = pack_bf16(a2, a3);
               }
+              tmem_st16(tR1 + lane_off + ch * 32, dd);
             }
             tc_wait_st();
             tc_fence_before();
@@ -357,40 +354,38 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           }
       }
       if (!ok) break;
-      // ---- item epilogue: dV, dK of key row r, columns 64*ch.. (D = 128) or 32*ch.. (D = 64)
+      // ---- item epilogue: dV, dK of key row r, columns (D/4)*ch ..
       ok = mbar_wait(bar_acc_full, ic & 1, ab, WAIT_BWD_ACC_FULL);
       if (!ok) break;
       tc_fence_after();
       const long long krow = ((long long)kv_tok0 + r) * p.h_kv + kvh;
       const bool to_fp32 = mode || p.causal_fp32;
-      constexpr int HALF = D / 2;
+      constexpr int QUART = D / 4;
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
+        const int col0 = ch * QUART;
+        uint32_t v[QUART];
+        if constexpr (D == 128) tmem_ld32((which ? tDK : tDV) + lane_off + col0, v);
+        else tmem_ld16((which ? tDK : tDV) + lane_off + col0, v);
+        tc_wait_ld();
+        if (key_valid) {
+          if (to_fp32) {
+            float4 *dst = reinterpret_cast<float4 *>((which ? p.dk_acc : p.dv_acc) + krow * D + col0);
 #pragma unroll
-        for (int c = 0; c < HALF / 32; ++c) {
-          const int col0 = ch * HALF + c * 32;
-          uint32_t v[32];
-          tmem_ld32((which ? tDK : tDV) + lane_off + col0, v);
-          tc_wait_ld();
-          if (key_valid) {
-            if (to_fp32) {
-              float4 *dst = reinterpret_cast<float4 *>((which ? p.dk_acc : p.dv_acc) + krow * D + col0);
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                float4 a = dst[i];
-                a.x += __uint_as_float(v[4 * i]); a.y += __uint_as_float(v[4 * i + 1]);
-                a.z += __uint_as_float(v[4 * i + 2]); a.w += __uint_as_float(v[4 * i + 3]);
-                dst[i] = a;
-              }
-            } else {
-              uint4 *dst = reinterpret_cast<uint4 *>((which ? p.dk_out : p.dv_out) + krow * D + col0);
-#pragma unroll
-              for (int i = 0; i < 4; ++i)
-                dst[i] = make_uint4(pack_bf16(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
-                                    pack_bf16(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
-                                    pack_bf16(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
-                                    pack_bf16(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
+            for (int i = 0; i < QUART / 4; ++i) {
+              float4 a = dst[i];
+              a.x += __uint_as_float(v[4 * i]); a.y += __uint_as_float(v[4 * i + 1]);
+              a.z += __uint_as_float(v[4 * i + 2]); a.w += __uint_as_float(v[4 * i + 3]);
+              dst[i] = a;
             }
+          } else {
+            uint4 *dst = reinterpret_cast<uint4 *>((which ? p.dk_out : p.dv_out) + krow * D + col0);
+#pragma unroll
+            for (int i = 0; i < QUART / 8; ++i)
+              dst[i] = make_uint4(pack_bf16(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
+                                  pack_bf16(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
+                                  pack_bf16(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
+                                  pack_bf16(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
           }
         }
       }
@@ -406,7 +401,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+  if (warp == 17) { tc_fence_after(); tmem_dealloc(tmem, 512); }
 }
 
 // Row statistics of the backward pass, stored per 128-row query tile:
