@@ -68,7 +68,7 @@ def peaks():
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture of this workload (the summary under
 # profiles/ gives the command); None for workloads that were not captured
-NCU_DRAM_BYTES = {("cfg2-7b-layer", "replay_bwd_dkdv"): 1.226e9, ("cfg2-7b-layer", "replay_bwd_dq"): 0.384e9,
+NCU_DRAM_BYTES = {("cfg2-7b-layer", "replay_bwd_dkdv"): 1.215e9, ("cfg2-7b-layer", "replay_bwd_dq"): 0.384e9,
                   ("cfg2-7b-layer", "replay_fwd"): 0.254e9}
 
 
