@@ -197,3 +197,17 @@ def run_forward_backward(plan: Plan, t, out):
                     out["dq_r"], out["dk_r"], out["dv_r"], out["dk_p"], out["dv_p"], out["ws"])
     plan.prefill_bwd(t["q_p"], t["k_p"], t["v_p"], out["o_p"], out["lse_p"], t["do_p"], out["dk_p"], out["dv_p"],
                      out["dq_p"], None, None, out["ws"])
+
+
+def capture_step(plan: Plan, t, out):
+    """The whole hot path captured once into a CUDA graph (the library allocates nothing and does not synchronise
+    in its launch path); `graph.replay()` then re-runs it on the same buffers.  Pays off for launch-bound sizes."""
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        run_forward_backward(plan, t, out)  # first use of each kernel sets its attributes: keep that out of the capture
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            run_forward_backward(plan, t, out)
+    torch.cuda.current_stream().wait_stream(s)
+    return g

@@ -110,3 +110,24 @@ def test_flattened_baseline_matches_tree(B):
         np.testing.assert_allclose(got["lse_p"][:, sl], ref["lse_r"][:, r_off:r_off + r], atol=pu.LSE_ABS)
         off += P + r; r_off += r
     pu.assert_parity({"dk_p": dk, "dv_p": dv, "dq_p": dq}, {k: ref[k] for k in ("dk_p", "dv_p", "dq_p")})
+
+
+def test_cuda_graph_replay_is_bitwise_the_eager_step(B):
+    """The four entry points capture into a CUDA graph (no allocation or synchronisation in the launch path)."""
+    w = _wl("graph", [256], [[128] * 4], 4, 4, 64, 61)
+    t = {k: v.cuda() for k, v in wl.make_tensors(w).items()}
+    plan = B.Plan(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, device=0, flags=B.FLAG_ZERO_PROMPT_GRAD)
+    out = B.alloc_outputs(plan)
+    B.run_forward_backward(plan, t, out)
+    torch.cuda.synchronize()
+    eager = {k: v.clone() for k, v in out.items() if k != "ws"}
+    g = B.capture_step(plan, t, out)
+    for k, v in out.items():
+        if k not in ("ws", "dk_p", "dv_p"):
+            v.fill_(float("nan"))
+    g.replay()
+    g.replay()
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0)
+    for k, v in eager.items():
+        assert torch.equal(v, out[k]), k
