@@ -12,8 +12,7 @@ enum WaitSite : int {
   WAIT_FWD_Q_FULL = 1, WAIT_FWD_Q_EMPTY = 2, WAIT_FWD_KV_FULL = 3, WAIT_FWD_KV_EMPTY = 4, WAIT_FWD_S_FULL = 5,
   WAIT_FWD_P_FULL = 6, WAIT_FWD_O_FULL = 7, WAIT_FWD_O_EMPTY = 8,
   WAIT_BWD_KV_FULL = 20, WAIT_BWD_KV_EMPTY = 21, WAIT_BWD_QDO_FULL = 22, WAIT_BWD_QDO_EMPTY = 23, WAIT_BWD_S_FULL = 24,
-  WAIT_BWD_PDS_FULL = 25, WAIT_BWD_MMA2 = 26, WAIT_BWD_DQ_FREE = 27, WAIT_BWD_ACC_FULL = 28, WAIT_BWD_ACC_EMPTY = 29, WAIT_BWD_ROWS = 30,
-  WAIT_DRAIN = 40
+  WAIT_BWD_PDS_FULL = 25, WAIT_BWD_ACC_FULL = 28, WAIT_BWD_ACC_EMPTY = 29
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -86,7 +85,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
 }
 
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---------------------------------------------------------------------- TMA
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, uint32_t bar, int c0, int c1, int c2) {
@@ -118,21 +116,6 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
-}
-
 // Instruction descriptor for kind::f16 with bf16 operands and fp32 accumulate.
 // Bits: [4,6) D format (1 = f32), [7,10) A format (1 = bf16), [10,13) B format,
 // 15 A major (1 = MN), 16 B major (1 = MN), [17,23) N >> 3, [24,29) M >> 4.
@@ -149,12 +132,7 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, int a_mn_major, 
 //  - MN-major operand (128-byte lines along M/N, one line per K index):
 //    leading offset = distance between 64-element chunks of M/N, stride
 //    offset = distance between groups of 8 K indices.
-__device__ __forceinline__ uint64_t make_sdesc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
-}
-
-// The same descriptor as two 32-bit words, so that the issuing thread only adds
+// It is built as two 32-bit words, so that the issuing thread only adds
 // a constant per K step: the high word depends on the layout alone, the low
 // word is address | LBO.
 __host__ __device__ constexpr uint32_t sdesc_hi(uint32_t sbo_bytes) { return (sbo_bytes >> 4) | (1u << 14) | (2u << 29); }
@@ -202,15 +180,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
@@ -302,9 +271,6 @@ __device__ __forceinline__ float ex2_fma(float x) {
   p = fmaf(p, f, 0.6931218504905701f);
   p = fmaf(p, f, 0.9999992847442627f);
   return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
-}
-__device__ __forceinline__ void red_add_v4(float *gptr, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(gptr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
 }  // namespace augtree
