@@ -1,4 +1,4 @@
-// Pack & schedule (host): prefix sums, work items for the four kernels and their
+// Pack & schedule (host): prefix sums, work items for the six schedules (forward, key-side and query-side backward; prefill and replay call) and their
 // largest-first assignment to replay lanes.
 //
 // Units and weights follow Sec. 3.4 ("Replay units and grid assignment"): a
