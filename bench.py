@@ -287,7 +287,11 @@ def main():
     per_kernel = {}
     for n, (tot, cnt) in zip(names, kt):
         if cnt:
-            per_kernel[n] = {"ms": tot / cnt, "tflops": fl[n] / (tot / cnt * 1e-3) / 1e12, "launches": cnt}
+            # tflops: the GEMM FLOPs the launch executes; tflops_algorithmic: its share of the 14 d per pair (the
+            # query-side kernel's S and dP are recomputation: only its dQ GEMM, 2 d of its 6 d, is algorithmic)
+            alg = fl[n] / 3 if n.endswith("_dq") else fl[n]
+            per_kernel[n] = {"ms": tot / cnt, "tflops": fl[n] / (tot / cnt * 1e-3) / 1e12,
+                             "tflops_algorithmic": alg / (tot / cnt * 1e-3) / 1e12, "launches": cnt}
     dom = max(per_kernel, key=lambda n: per_kernel[n]["ms"])
     roofline = {"bound": "tensor", "kernel": f"{kfun[dom]} ({dom})", "achieved": per_kernel[dom]["tflops"],
                 "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": per_kernel[dom]["tflops"] / pk["bf16_tflops"],
