@@ -23,6 +23,16 @@
  *  - Row a of a sequence sees keys b <= a (inclusive diagonal).
  *  - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous; they
  *    return after enqueueing.  Nothing is allocated or freed per call.
+ *  - A plan belongs to the device given to augtree_plan_create.  The five
+ *    launching entry points (prefill/replay, fwd/bwd, and the static-scratch
+ *    forward) must be called with that device current in the calling thread
+ *    and with a stream of that device; with another device current they
+ *    return AUGTREE_ERR_INVALID_ARG and launch nothing.  One process may hold
+ *    plans for several devices and use them from several threads; a plan is
+ *    immutable after creation, and concurrent calls on one plan are safe as
+ *    long as each has its own workspace.  Plan creation, destruction and the
+ *    status and timing queries switch to the plan's device themselves and
+ *    restore the caller's.
  *  - Every function returns AUGTREE_OK (0) or a negative augtree_status code;
  *    the library never aborts, traps or throws.  Errors detected on the
  *    device (a bounded wait that ran out) are recorded in a status word that

@@ -1,7 +1,11 @@
 """Independent restatement of the pack-and-schedule metadata (test infrastructure only).
 
 Written from the rules, not from the library's source: the tests demand that
-the library's tables equal these bit for bit.
+the library's tables equal these bit for bit.  What pins THESE tables is not
+the library but tests/test_packing_cover.py: every item is expanded from its
+fields into the (query, key, head) triples it stands for, and each schedule
+must cover the tree mask of Eq. 1 exactly once, with weights equal to visited
+tile counts and one owner per prompt-KV tile.
 
 Rules.  Tiles are 128 query rows by 128 keys.  A forward item is one (pair of
 consecutive query tiles, query head[, prompt-KV shard]); its weight is the

@@ -29,7 +29,7 @@ LSE is [H_q, tokens], natural log of the scaled scores' sum of exponentials
 (LSE = m + ln l in the (m, l, O_acc) notation of Sec. 3.3).
 Query head h reads KV head h // (H_q / H_kv).
 
-Parity pins (tests/test_oracle_*.py): central finite differences, the dense
+Parity pins (tests/test_oracle_pins.py): central finite differences, the dense
 tree-mask formulation, split + merge of partial softmax states, torch's
 scaled_dot_product_attention for G = 1, closed forms (zero keys, constant
 values, first row), and row-sum invariants.  Every function below is covered
@@ -282,6 +282,87 @@ def dkv_key(tb, q_p, k_p, v_p, do_p, q_r, k_r, v_r, do_r, kind, token, kv_head):
             dv += p_ab * do
             ds = p_ab * (do @ vvec - do @ o)
             dk += tb.scale * ds * q
+    return dk, dv
+
+
+def dkv_keys_block(tb, q_p, k_p, v_p, do_p, q_r, k_r, v_r, do_r, kind, tokens, kv_head, block=256):
+    """dK and dV of several keys of ONE sequence part (all `tokens` prompt tokens of one group, kind 'p',
+    or response tokens of one branch, kind 'r') and one KV head: the sums of dkv_key, taken a block of
+    query rows at a time so that each row's softmax over its full visible key set is one matrix product.
+
+    Rows that see a prompt key: the prompt rows from the key on, and every response row of every branch
+    of the group (Eq. 2).  Rows that see a response key: the rows of its branch from the key on.
+    Returns (dk [len(tokens), d], dv [len(tokens), d]).  Same formulas as dkv_key; pinned against it.
+    """
+    hq, hkv, scale = tb.h_q, tb.h_kv, tb.scale
+    rep = hq // hkv
+    tokens = [int(x) for x in tokens]
+    f = lambda x: np.asarray(x, dtype=np.float64)
+    if kind == "p":
+        g = int(np.searchsorted(tb.cu_p, tokens[0], side="right") - 1)
+        seq0, seq1 = int(tb.cu_p[g]), int(tb.cu_p[g + 1])
+        branches = range(int(tb.cu_b[g]), int(tb.cu_b[g + 1]))
+    else:
+        b = int(np.searchsorted(tb.cu_r, tokens[0], side="right") - 1)
+        g = int(np.searchsorted(tb.cu_b, b, side="right") - 1)
+        seq0, seq1 = int(tb.cu_r[b]), int(tb.cu_r[b + 1])
+        branches = []
+    assert all(seq0 <= t < seq1 for t in tokens), "keys must lie in one prompt / one branch"
+    p0, p1 = int(tb.cu_p[g]), int(tb.cu_p[g + 1])
+    kp, vp = f(k_p[p0:p1, kv_head]), f(v_p[p0:p1, kv_head])
+    key_pos = np.asarray([t - seq0 for t in tokens])           # position inside the key's own sequence part
+    dk, dv = np.zeros((len(tokens), tb.head_dim)), np.zeros((len(tokens), tb.head_dim))
+
+    def rows_block(q, do, keys_k, keys_v, first_pos, own_len, sel_cols, sel_visible):
+        """q, do: [m, d] rows at positions first_pos.. of a causal range of own_len keys that follows an
+        unmasked range; keys_*: [unmasked + own_len, d]; adds the rows' terms for the key columns sel_cols
+        (sel_visible[m, n_sel]: whether row sees that key)."""
+        m = q.shape[0]
+        n_un = keys_k.shape[0] - own_len
+        s = scale * (q @ keys_k.T)
+        pos = first_pos + np.arange(m)
+        col = np.arange(keys_k.shape[0])
+        s = np.where(col[None, :] <= n_un + pos[:, None], s, -np.inf)
+        mx = s.max(axis=1, keepdims=True)
+        e = np.exp(s - mx)
+        p = e / e.sum(axis=1, keepdims=True)
+        o = p @ keys_v
+        delta = (do * o).sum(axis=1)
+        inside = sel_cols < keys_k.shape[0]          # a key past the block's last row is in no row's range
+        cols = np.where(inside, sel_cols, 0)
+        psel = np.where(sel_visible & inside[None, :], p[:, cols], 0.0)             # [m, n_sel]
+        dsel = psel * (do @ keys_v[cols].T - delta[:, None])
+        return scale * (dsel.T @ q), psel.T @ do
+
+    for h in range(kv_head * rep, (kv_head + 1) * rep):
+        if kind == "p":
+            # later prompt rows of the same prompt (causal inside the prompt)
+            lo = int(key_pos.min())
+            for a0 in range(lo, p1 - p0, block):
+                a1 = min(a0 + block, p1 - p0)
+                vis = (a0 + np.arange(a1 - a0))[:, None] >= key_pos[None, :]
+                ddk, ddv = rows_block(f(q_p[p0 + a0:p0 + a1, h]), f(do_p[p0 + a0:p0 + a1, h]), kp[:a1], vp[:a1], a0, a1, key_pos, vis)
+                dk += ddk; dv += ddv
+            # every response row of every branch of the group (unmasked on the prompt)
+            for bi in branches:
+                r0, r1 = int(tb.cu_r[bi]), int(tb.cu_r[bi + 1])
+                kr, vr = f(k_r[r0:r1, kv_head]), f(v_r[r0:r1, kv_head])
+                for a0 in range(0, r1 - r0, block):
+                    a1 = min(a0 + block, r1 - r0)
+                    kk, vv = np.concatenate([kp, kr[:a1]]), np.concatenate([vp, vr[:a1]])
+                    vis = np.ones((a1 - a0, len(tokens)), dtype=bool)
+                    ddk, ddv = rows_block(f(q_r[r0 + a0:r0 + a1, h]), f(do_r[r0 + a0:r0 + a1, h]), kk, vv, a0, a1, key_pos, vis)
+                    dk += ddk; dv += ddv
+        else:
+            kr, vr = f(k_r[seq0:seq1, kv_head]), f(v_r[seq0:seq1, kv_head])
+            lo = int(key_pos.min())
+            for a0 in range(lo, seq1 - seq0, block):
+                a1 = min(a0 + block, seq1 - seq0)
+                kk, vv = np.concatenate([kp, kr[:a1]]), np.concatenate([vp, vr[:a1]])
+                vis = (a0 + np.arange(a1 - a0))[:, None] >= key_pos[None, :]
+                ddk, ddv = rows_block(f(q_r[seq0 + a0:seq0 + a1, h]), f(do_r[seq0 + a0:seq0 + a1, h]), kk, vv, a0, a1,
+                                      (p1 - p0) + key_pos, vis)
+                dk += ddk; dv += ddv
     return dk, dv
 
 

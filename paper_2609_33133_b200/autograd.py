@@ -5,7 +5,9 @@ response tokens of a plan's groups; backward fills the gradients of all six inpu
 backward is the one the method requires (Sec. 3.2): the replay backward first, which seeds the shared
 prompt-KV gradient with the sum over every branch (Eq. 2), then the prefill backward, which adds the
 prompt's own contribution and pushes the total through the prefill pass.  Inputs and outputs are bf16
-`[tokens, heads, head_dim]`; the prompt-KV gradients are accumulated in fp32 and cast once at the end.
+`[tokens, heads, head_dim]`; the prompt-KV gradients are accumulated in fp32 and cast once at the end
+(autograd hands a gradient back in its input's dtype).  The fp32 accumulators of the latest backward stay
+available as `plan.prompt_grad_fp32 = (dK_P, dV_P)` for callers that want them unrounded.
 """
 from __future__ import annotations
 
@@ -52,6 +54,7 @@ class _TreeAttention(torch.autograd.Function):
         dv_p = torch.empty((plan.total_p, hkv, d), device=dev, dtype=bf)
         plan.replay_bwd(q_r, k_r, v_r, k_p, v_p, o_r, lse_r, do_r, dq_r, dk_r, dv_r, dk_acc, dv_acc, ws)
         plan.prefill_bwd(q_p, k_p, v_p, o_p, lse_p, do_p, dk_acc, dv_acc, dq_p, dk_p, dv_p, ws)
+        plan.prompt_grad_fp32 = (dk_acc, dv_acc)
         return None, dq_p, dk_p, dv_p, dq_r, dk_r, dv_r
 
 

@@ -100,12 +100,6 @@ int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long 
   p.items = s.d_items; p.lane_ptr = s.d_lane_ptr;
   p.o = static_cast<__nv_bfloat16 *>(o); p.lse = lse; p.part_o = part_o; p.part_lse = part_lse;
   p.n_tok = q_tok; p.h_q = pl->h_q; p.scale_log2 = pl->scale * 1.4426950408889634f; p.status = pl->d_status;
-  static bool attr_set[2] = {false, false};
-  if (!attr_set[D / 128]) {
-    if (cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kBytes) != cudaSuccess)
-      return AUGTREE_ERR_CUDA;
-    attr_set[D / 128] = true;
-  }
   const int kind = (int)(&s - pl->sched);
   timing_mark(pl, kind, false, st);
   fwd_kernel<D><<<pl->n_lanes, kFwdThreads, FwdSmem<D>::kBytes, st>>>(mq, mka, mva, mkb, mvb, p);
@@ -157,12 +151,6 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     p.dk_acc = a.dk_acc; p.dv_acc = a.dv_acc; p.n_tiles = a.n_tiles; p.h_q = pl->h_q; p.h_kv = pl->h_kv;
     p.causal_fp32 = a.causal_fp32; p.scale = pl->scale; p.scale_log2 = pl->scale * 1.4426950408889634f;
     p.status = pl->d_status;
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[D / 128]) {
-      if (cudaFuncSetAttribute(bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kBytes) != cudaSuccess)
-        return AUGTREE_ERR_CUDA;
-      attr_set[D / 128] = true;
-    }
     const int kind = (int)(&s - pl->sched);
     timing_mark(pl, kind, false, st);
     bwd_kernel<D><<<pl->n_lanes, kBwdThreads, BwdSmem<D>::kBytes, st>>>(mq, mdo, mk0, mv0, mk1, mv1, p);
@@ -178,12 +166,6 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     p.items = a.dq_sched->d_items; p.lane_ptr = a.dq_sched->d_lane_ptr; p.stats = stats;
     p.dq = static_cast<__nv_bfloat16 *>(a.dq); p.n_tiles = a.n_tiles; p.h_q = pl->h_q;
     p.scale = pl->scale; p.scale_log2 = pl->scale * 1.4426950408889634f; p.status = pl->d_status;
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[D / 128]) {
-      if (cudaFuncSetAttribute(dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<D>::kBytes) != cudaSuccess)
-        return AUGTREE_ERR_CUDA;
-      attr_set[D / 128] = true;
-    }
     const int kind = (int)(a.dq_sched - pl->sched);
     timing_mark(pl, kind, false, st);
     // causal keys come from the queries' own sequence tensor (k0/v0)
@@ -206,8 +188,30 @@ void timing_mark(const augtree_plan *pl, int kind, bool stop, cudaStream_t st) {
   ++u;
 }
 
+// Launch entry points: the plan must live on a device, and that device must be the calling thread's current
+// one (tensor maps are encoded and kernels launched in the current context).
 int check_plan(const augtree_plan *pl) {
   if (!pl || pl->device < 0 || pl->n_lanes < 1) return AUGTREE_ERR_INVALID_ARG;
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess) return AUGTREE_ERR_CUDA;
+  if (cur != pl->device) return AUGTREE_ERR_INVALID_ARG;
+  return AUGTREE_OK;
+}
+
+// Queries that only read plan state: any current device will do.
+int check_plan_any_device(const augtree_plan *pl) {
+  if (!pl || pl->device < 0 || pl->n_lanes < 1) return AUGTREE_ERR_INVALID_ARG;
+  return AUGTREE_OK;
+}
+
+// The tile kernels use more than the default 48 KB of dynamic shared memory.  The attribute belongs to
+// the (function, device) pair, so it is set for the plan's device at plan creation, with that device current.
+template <int D>
+int set_kernel_attributes() {
+  if (cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<D>::kBytes) != cudaSuccess)
+    return AUGTREE_ERR_CUDA;
   return AUGTREE_OK;
 }
 
@@ -243,7 +247,12 @@ int augtree_plan_create(const augtree_desc_t *desc, int device, augtree_plan_t *
     int prev = 0;
     cudaGetDevice(&prev);
     r = cudaSetDevice(device) == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
-    for (int k = 0; k < SCHED_COUNT && !r; ++k) r = upload_sched(pl->sched[k], pl->n_lanes);
+    if (!r) r = pl->head_dim == 128 ? set_kernel_attributes<128>() : set_kernel_attributes<64>();
+    try {
+      for (int k = 0; k < SCHED_COUNT && !r; ++k) r = upload_sched(pl->sched[k], pl->n_lanes);
+    } catch (...) {
+      r = AUGTREE_ERR_INTERNAL;
+    }
     if (!r) r = upload(pl->seg_replay, &pl->d_seg_replay);
     if (!r) r = upload(pl->seg_prefill, &pl->d_seg_prefill);
     if (!r) r = upload(pl->branch_group, &pl->d_branch_group);
@@ -452,7 +461,7 @@ int augtree_prefill_bwd(const augtree_plan_t *pl, const void *q_p, const void *k
 }
 
 int augtree_last_device_status(const augtree_plan_t *pl, int *status, int *detail) {
-  int r = check_plan(pl);
+  int r = check_plan_any_device(pl);
   if (r || !status) return AUGTREE_ERR_INVALID_ARG;
   int prev = 0;
   cudaGetDevice(&prev);
@@ -469,7 +478,7 @@ int augtree_last_device_status(const augtree_plan_t *pl, int *status, int *detai
 }
 
 int augtree_set_timing(augtree_plan_t *pl, int enable) {
-  int r = check_plan(pl);
+  int r = check_plan_any_device(pl);
   if (r) return r;
   int prev = 0;
   cudaGetDevice(&prev);
@@ -491,7 +500,7 @@ int augtree_set_timing(augtree_plan_t *pl, int enable) {
 }
 
 int augtree_get_kernel_time(const augtree_plan_t *pl, int kernel, float *total_ms, int *launches) {
-  int r = check_plan(pl);
+  int r = check_plan_any_device(pl);
   if (r || kernel < 0 || kernel >= SCHED_COUNT || !total_ms || !launches) return AUGTREE_ERR_INVALID_ARG;
   *total_ms = 0.f; *launches = 0;
   const Timing *t = pl->timing;

@@ -95,9 +95,9 @@ struct ExactGrid {
 
 }  // namespace
 
-extern "C" int augtree_assign_grid(const int64_t *weight, const int64_t *size, int n_units, int n_rounds, int n_lanes,
-                                   int64_t cell_cap, int exact_max_units, int32_t *round_out, int32_t *lane_out,
-                                   int64_t *critical_path, int32_t *solved_exactly) {
+static int assign_grid_impl(const int64_t *weight, const int64_t *size, int n_units, int n_rounds, int n_lanes,
+                            int64_t cell_cap, int exact_max_units, int32_t *round_out, int32_t *lane_out,
+                            int64_t *critical_path, int32_t *solved_exactly) {
   if (n_units < 0 || n_rounds < 1 || n_lanes < 1 || (n_units > 0 && (!weight || !round_out || !lane_out))) return AUGTREE_ERR_INVALID_ARG;
   if (cell_cap > 0 && !size && n_units > 0) return AUGTREE_ERR_INVALID_ARG;
   if (n_rounds > 1024 || n_lanes > 65536) return AUGTREE_ERR_UNSUPPORTED;
@@ -125,22 +125,28 @@ extern "C" int augtree_assign_grid(const int64_t *weight, const int64_t *size, i
     std::vector<int32_t> ids(n_units);
     std::iota(ids.begin(), ids.end(), 0);
     std::stable_sort(ids.begin(), ids.end(), [&](int32_t a, int32_t c) { return weight[a] > weight[c]; });
-    std::vector<int64_t> load((size_t)n_rounds * n_lanes, 0), used((size_t)n_rounds * n_lanes, 0), peak(n_rounds, 0);
+    // Empty cells of a round are interchangeable and the lowest lane wins ties, so the occupied lanes of a
+    // round are always a prefix 0 .. filled-1: only those and the first empty one are candidates, and only
+    // those are stored (the grid itself may be far larger than the number of units).
+    std::vector<std::vector<int64_t>> load(n_rounds), used(n_rounds);
+    std::vector<int64_t> peak(n_rounds, 0);
     for (int32_t k : ids) {
       int bt = -1, bj = -1;
       int64_t b_grow = 0, b_new = 0;
-      for (int t = 0; t < n_rounds; ++t)
-        for (int j = 0; j < n_lanes; ++j) {
-          const size_t c = (size_t)t * n_lanes + j;
-          if (cell_cap > 0 && used[c] + size[k] > cell_cap) continue;
-          const int64_t nw = load[c] + weight[k], grow = std::max(peak[t], nw) - peak[t];
+      for (int t = 0; t < n_rounds; ++t) {
+        const int filled = (int)load[t].size();
+        for (int j = 0; j < std::min(filled + 1, n_lanes); ++j) {
+          const int64_t have = j < filled ? load[t][j] : 0, mem = j < filled ? used[t][j] : 0;
+          if (cell_cap > 0 && mem + size[k] > cell_cap) continue;
+          const int64_t nw = have + weight[k], grow = std::max(peak[t], nw) - peak[t];
           if (bt < 0 || grow < b_grow || (grow == b_grow && nw < b_new)) { bt = t; bj = j; b_grow = grow; b_new = nw; }
         }
+      }
       if (bt < 0) return AUGTREE_ERR_UNSUPPORTED;
-      const size_t c = (size_t)bt * n_lanes + bj;
-      load[c] += weight[k];
-      if (size) used[c] += size[k];
-      peak[bt] = std::max(peak[bt], load[c]);
+      if (bj == (int)load[bt].size()) { load[bt].push_back(0); used[bt].push_back(0); }
+      load[bt][bj] += weight[k];
+      if (size) used[bt][bj] += size[k];
+      peak[bt] = std::max(peak[bt], load[bt][bj]);
       round_out[k] = bt;
       lane_out[k] = bj;
     }
@@ -149,4 +155,17 @@ extern "C" int augtree_assign_grid(const int64_t *weight, const int64_t *size, i
   if (critical_path) *critical_path = path;
   if (solved_exactly) *solved_exactly = exact ? 1 : 0;
   return AUGTREE_OK;
+}
+
+// Nothing may leave through the C interface but a status code: a failed allocation inside the solvers
+// (std::bad_alloc) is reported as AUGTREE_ERR_INTERNAL.
+extern "C" int augtree_assign_grid(const int64_t *weight, const int64_t *size, int n_units, int n_rounds, int n_lanes,
+                                   int64_t cell_cap, int exact_max_units, int32_t *round_out, int32_t *lane_out,
+                                   int64_t *critical_path, int32_t *solved_exactly) {
+  try {
+    return assign_grid_impl(weight, size, n_units, n_rounds, n_lanes, cell_cap, exact_max_units, round_out, lane_out,
+                            critical_path, solved_exactly);
+  } catch (...) {
+    return AUGTREE_ERR_INTERNAL;
+  }
 }

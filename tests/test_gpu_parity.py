@@ -40,13 +40,11 @@ def test_small_cases_match_oracle(B, w):
     t = wl.make_tensors(w)
     got, _ = pu.run_gpu(B, w, t)
     if w.name == "tiny":
-        # One query row over two keys: the relative-L2 figure is a statistic over a
-        # tensor and does not average on 64 numbers (bf16 rounding of O, P and dS is
-        # 2^-9 per element and the two-key softmax backward cancels).  The absolute
-        # bound is kept; the relative one is widened for this degenerate case only.
-        rows = pu.errors(got, pu.run_oracle(w, t))
-        for k, (rel, mx, finite) in rows.items():
-            assert finite and mx <= (pu.LSE_ABS if k.startswith("lse") else pu.MAX_ABS) and rel <= 3e-2, (k, rel, mx)
+        # One query row over two keys, 64 numbers per tensor: the relative-L2 figure is a statistic over a
+        # tensor and does not average here (bf16 rounding of O, P and dS is 2^-9 per element and the two-key
+        # softmax backward cancels).  Measured 1.3e-2; bound for this case only 3e-2.  The absolute bounds stay.
+        wide = {k: {"rel_l2": 3e-2} for k in ("o_p", "o_r", *pu.GRADS)}
+        pu.assert_parity(got, pu.run_oracle(w, t), exceptions=wide)
         return
     pu.assert_parity(got, pu.run_oracle(w, t))
 

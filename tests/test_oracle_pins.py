@@ -219,6 +219,24 @@ def test_key_form_matches_matrix_form():
         np.testing.assert_allclose(dv, res["dv" + sfx][tok, c], rtol=1e-10, atol=1e-11)
 
 
+def test_key_block_form_matches_key_form_and_matrix_form():
+    """The row-block form (several keys, query rows a block at a time) against the per-key row form and the
+    n x n matrix form, with blocks that cut through the prompt, through branches and behind the keys."""
+    tb, t = _rand_tree(12, [9, 5], [[6, 1, 4], [3]], 4, 2, 8)
+    res = _run(tb, t)
+    a = [t[n] for n in ("q_p", "k_p", "v_p", "do_p", "q_r", "k_r", "v_r", "do_r")]
+    for kind, toks, c in [("p", [0, 3, 8], 0), ("p", [9, 13], 1), ("r", [0, 5], 1), ("r", [7, 10], 0), ("r", [11, 13], 1), ("r", [6], 0)]:
+        for block in (4, 256):
+            dk, dv = ora.dkv_keys_block(tb, *a, kind, toks, c, block=block)
+            sfx = "_p" if kind == "p" else "_r"
+            for i, tok in enumerate(toks):
+                k1, v1 = ora.dkv_key(tb, *a, kind, tok, c)
+                np.testing.assert_allclose(dk[i], k1, rtol=1e-11, atol=1e-12)
+                np.testing.assert_allclose(dv[i], v1, rtol=1e-11, atol=1e-12)
+                np.testing.assert_allclose(dk[i], res["dk" + sfx][tok, c], rtol=1e-10, atol=1e-11)
+                np.testing.assert_allclose(dv[i], res["dv" + sfx][tok, c], rtol=1e-10, atol=1e-11)
+
+
 # --- work accounting: flattening repeats the prompt pairs G times (Sec. 1) ---
 def test_redundancy_fraction():
     for G, want in [(8, 0.875), (64, 0.984375)]:

@@ -6,7 +6,7 @@ They cannot supply the workspace the sharded forward needs, so this entry point 
 32 MiB array inside the library's device image.  The test calls it through the C interface twice in a row
 and checks each result against the ordinary entry point (which gets a torch-allocated workspace) with the
 tolerances of the other parity tests; the two paths run the same kernels, so they also agree bit for bit.
-It also checks that free device memory does not move across a call and that an oversized plan is refused.
+Each result is also compared with the fp64 oracle directly.  It also checks that free device memory does not move across a call and that an oversized plan is refused.
 """
 import numpy as np
 import pytest
@@ -57,10 +57,13 @@ def test_static_scratch_matches_workspace_variant_twice(B):
         torch.cuda.synchronize()
         assert torch.cuda.mem_get_info()[0] == free1, "the call changed the amount of free device memory"
         got_o2, got_lse2 = o.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+        oracle = pu.run_oracle(w, wl.make_tensors(w))
+        oracle = {"o_r": oracle["o_r"], "lse_r": oracle["lse_r"]}
         for go, gl in ((got_o, got_lse), (got_o2, got_lse2)):
             rows = pu.errors({"o_r": go, "lse_r": gl}, {"o_r": ref_o, "lse_r": ref_lse})
             assert rows["o_r"][0] <= pu.REL_L2 and rows["o_r"][1] <= pu.MAX_ABS and rows["lse_r"][1] <= pu.LSE_ABS, rows
             assert np.array_equal(go, ref_o) and np.array_equal(gl, ref_lse)
+            pu.assert_parity({"o_r": go, "lse_r": gl}, oracle)
 
 
 def test_static_scratch_refuses_oversized_plan(B):
