@@ -125,7 +125,13 @@ enum {
 int augtree_plan_create(const augtree_desc_t *desc, int device, augtree_plan_t **out);
 int augtree_plan_destroy(augtree_plan_t *plan);
 
-/* Bytes of caller-provided scratch the forward and backward calls need. */
+/*
+ * Bytes of caller-provided scratch the forward and backward calls need.  Both
+ * forward calls need at least 256 bytes (the largest key norm per KV head,
+ * from which the tile kernel bounds the scores of a row), the sharded replay
+ * forward also room for the shards' partial states; the backward calls need
+ * the per-row statistics.
+ */
 int augtree_plan_workspace_bytes(const augtree_plan_t *plan, size_t *fwd_bytes, size_t *bwd_bytes);
 
 /*
@@ -154,6 +160,7 @@ int augtree_plan_metadata(const augtree_plan_t *plan, int table_id, void *host_d
  * attention of every prompt on itself.  k_p/v_p are only read and stay where
  * they are for the replay calls.
  *   q_p [sumP,H_q,d]  k_p,v_p [sumP,H_kv,d]  ->  o_p [sumP,H_q,d] bf16, lse_p [H_q,sumP] fp32
+ * ws: fwd_bytes of scratch (augtree_plan_workspace_bytes), else AUGTREE_ERR_WORKSPACE.
  */
 int augtree_prefill_fwd(const augtree_plan_t *plan, const void *q_p, const void *k_p, const void *v_p,
                         void *o_p, float *lse_p, void *ws, size_t ws_bytes, void *stream);
@@ -220,13 +227,14 @@ int augtree_prefill_bwd(const augtree_plan_t *plan, const void *q_p, const void 
  *
  *  - A plan whose forward scratch need (augtree_plan_workspace_bytes, fwd)
  *    exceeds the array is refused with AUGTREE_ERR_WORKSPACE; nothing is
- *    launched.  Plans without prompt-KV shards need no scratch and always fit.
+ *    launched.  Plans without prompt-KV shards need 256 bytes and always fit.
  *  - The first call on each device looks up the array's device address (a
  *    one-off set-up step, done with that device current).  Make that first
  *    call outside any stream capture.
  *  - All calls on a device share the one array and it keeps whatever the last
- *    call left there.  Nothing in it has to start at zero: every value the
- *    merge kernel reads is written by the same call's tile kernel first.  Two
+ *    call left there.  The one part that must start at zero (the key-norm
+ *    maxima at its head) is cleared by every call on its stream; every other
+ *    value read is written by the same call first.  Two
  *    calls that may overlap on the GPU (different streams, no dependency) race
  *    on it; order them.
  * Arguments and results are those of augtree_replay_fwd.

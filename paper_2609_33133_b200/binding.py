@@ -14,7 +14,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libaugtree.so")
+LIB_PATH = os.environ.get("AUGTREE_LIB") or os.path.join(_HERE, "libaugtree.so")   # AUGTREE_LIB: another build of the library
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_33133_b200.build`")
 lib = C.CDLL(LIB_PATH)

@@ -2,6 +2,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstring>
 #include <mutex>
@@ -60,6 +61,8 @@ int make_map(CUtensorMap *m, const void *ptr, long long tokens, int heads, int d
   return r == CUDA_SUCCESS ? AUGTREE_OK : AUGTREE_ERR_CUDA;
 }
 
+constexpr size_t kFwdHeaderBytes = 256;  // head of the forward scratch: per-KV-head key-norm maxima (plan.cpp reserves it)
+
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 size_t al256(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -87,8 +90,20 @@ void timing_mark(const augtree_plan *pl, int kind, bool stop, cudaStream_t st);
 template <int D>
 int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long q_tok, const void *ka, const void *va,
                long long a_tok, const void *kb, const void *vb, long long b_tok, void *o, float *lse, float *part_o,
-               float *part_lse, cudaStream_t st) {
+               float *part_lse, void *ws, cudaStream_t st) {
   if (s.n_items() == 0) return AUGTREE_OK;
+  // first 256 bytes of the scratch: largest squared key norm per KV head (score bound of the tile kernel)
+  unsigned int *kmax2 = static_cast<unsigned int *>(ws);
+  if (cudaMemsetAsync(kmax2, 0, (size_t)pl->h_kv * sizeof(unsigned int), st) != cudaSuccess) return AUGTREE_ERR_CUDA;
+  {
+    const bool same = ka == kb;
+    const long long rows = a_tok + (same ? 0 : b_tok);
+    const unsigned blocks = (unsigned)std::min<long long>(296, std::max<long long>(1, rows / 64));
+    key_norm_kernel<D><<<dim3(blocks, (unsigned)pl->h_kv), 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(ka), a_tok,
+                                                                       static_cast<const __nv_bfloat16 *>(kb), same ? 0 : b_tok,
+                                                                       pl->h_kv, kmax2);
+    ++g_launches;
+  }
   CUtensorMap mq, mka, mva, mkb, mvb;
   int r;
   if ((r = make_map(&mq, q, q_tok, pl->h_q, D))) return r;
@@ -100,6 +115,7 @@ int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long 
   p.items = s.d_items; p.lane_ptr = s.d_lane_ptr;
   p.o = static_cast<__nv_bfloat16 *>(o); p.lse = lse; p.part_o = part_o; p.part_lse = part_lse;
   p.n_tok = q_tok; p.h_q = pl->h_q; p.scale_log2 = pl->scale * 1.4426950408889634f; p.status = pl->d_status;
+  p.kmax2 = reinterpret_cast<const float *>(kmax2);
   const int kind = (int)(&s - pl->sched);
   timing_mark(pl, kind, false, st);
   fwd_kernel<D><<<pl->n_lanes, kFwdThreads, FwdSmem<D>::kBytes, st>>>(mq, mka, mva, mkb, mvb, p);
@@ -330,16 +346,16 @@ int augtree_plan_metadata(const augtree_plan_t *pl, int table_id, void *host_dst
 
 int augtree_prefill_fwd(const augtree_plan_t *pl, const void *q_p, const void *k_p, const void *v_p, void *o_p,
                         float *lse_p, void *ws, size_t ws_bytes, void *stream) {
-  (void)ws; (void)ws_bytes;
   int r = check_plan(pl);
   if (r) return r;
   if (!q_p || !k_p || !v_p || !o_p || !lse_p) return AUGTREE_ERR_INVALID_ARG;
   if (!aligned16(q_p) || !aligned16(k_p) || !aligned16(v_p) || !aligned16(o_p)) return AUGTREE_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < kFwdHeaderBytes || !aligned16(ws)) return AUGTREE_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Sched &s = pl->sched[SCHED_PREFILL_FWD];
   if (pl->head_dim == 128)
-    return launch_fwd<128>(pl, s, q_p, pl->total_p, k_p, v_p, pl->total_p, k_p, v_p, pl->total_p, o_p, lse_p, nullptr, nullptr, st);
-  return launch_fwd<64>(pl, s, q_p, pl->total_p, k_p, v_p, pl->total_p, k_p, v_p, pl->total_p, o_p, lse_p, nullptr, nullptr, st);
+    return launch_fwd<128>(pl, s, q_p, pl->total_p, k_p, v_p, pl->total_p, k_p, v_p, pl->total_p, o_p, lse_p, nullptr, nullptr, ws, st);
+  return launch_fwd<64>(pl, s, q_p, pl->total_p, k_p, v_p, pl->total_p, k_p, v_p, pl->total_p, o_p, lse_p, nullptr, nullptr, ws, st);
 }
 
 int augtree_replay_fwd(const augtree_plan_t *pl, const void *q_r, const void *k_r, const void *v_r, const void *k_p,
@@ -351,18 +367,18 @@ int augtree_replay_fwd(const augtree_plan_t *pl, const void *q_r, const void *k_
   if (!aligned16(q_r) || !aligned16(k_r) || !aligned16(v_r) || !aligned16(k_p) || !aligned16(v_p) || !aligned16(o_r))
     return AUGTREE_ERR_INVALID_ARG;
   float *part_o = nullptr, *part_lse = nullptr;
+  if (!ws || ws_bytes < pl->ws_fwd || !aligned16(ws)) return AUGTREE_ERR_WORKSPACE;
   if (pl->max_splits > 1) {
-    if (!ws || ws_bytes < pl->ws_fwd || !aligned16(ws)) return AUGTREE_ERR_WORKSPACE;
-    part_o = static_cast<float *>(ws);
-    part_lse = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) +
+    part_o = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) + kFwdHeaderBytes);
+    part_lse = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) + kFwdHeaderBytes +
                                          al256((size_t)pl->max_splits * (size_t)pl->total_r * pl->h_q * pl->head_dim * 4));
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Sched &s = pl->sched[SCHED_REPLAY_FWD];
   if (pl->head_dim == 128)
-    r = launch_fwd<128>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, o_r, lse_r, part_o, part_lse, st);
+    r = launch_fwd<128>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, o_r, lse_r, part_o, part_lse, ws, st);
   else
-    r = launch_fwd<64>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, o_r, lse_r, part_o, part_lse, st);
+    r = launch_fwd<64>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, o_r, lse_r, part_o, part_lse, ws, st);
   if (r || pl->max_splits == 1) return r;
   // groups that ended up with one shard wrote their final output directly; the
   // merge kernel only touches tokens whose group has more than one shard
@@ -517,6 +533,15 @@ int augtree_get_kernel_time(const augtree_plan_t *pl, int kernel, float *total_m
 }
 
 long long augtree_launch_count(void) { return g_launches.load(); }
+
+#if AUGTREE_TRACE
+// Measurement build only (not declared in the public header): reads and clears the forward kernel's phase counters.
+int augtree_debug_fwd_trace(unsigned long long *out8) {
+  unsigned long long z[8] = {};
+  if (cudaMemcpyFromSymbol(out8, g_fwd_trace, sizeof(z)) != cudaSuccess) return AUGTREE_ERR_CUDA;
+  return cudaMemcpyToSymbol(g_fwd_trace, z, sizeof(z)) == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+}
+#endif
 
 const char *augtree_status_string(int s) {
   switch (s) {

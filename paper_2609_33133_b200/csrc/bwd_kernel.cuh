@@ -8,7 +8,7 @@
 // dq_kernel, query-stationary, so that neither side needs atomics.)
 //
 // Per (KV tile, Q tile, head) pair T, with S^T = K Q^T so that a TMEM lane is a key:
-//   P^T  = exp2(S^T * scale*log2e - lse2[q])          (element-wise warps)
+//   P^T  = exp2(S^T * scale*log2e - lse2[q])          (element-wise warps; packed fp32 arithmetic)
 //   dP^T = V dO^T
 //   dS^T = P^T * (scale*dP^T - scale*delta[q])        (element-wise warps)
 //   dV  += P^T dO      (A = P^T from TMEM)
@@ -32,7 +32,7 @@ struct BwdParams {
   const int32_t *items;     // lane order, 8 ints each
   const int32_t *lane_ptr;  // [gridDim.x + 1]
   const int32_t *segs;      // [n_seg][3] {first query token, length, first tile index}
-  const float *stats;       // [h_q][n_tiles][2][128]: lse*log2e (inf past the end), scale*rowsum(dO*O)
+  const float *stats;       // [h_q][n_tiles][2][128]: -lse*log2e (-inf past the end), -scale*rowsum(dO*O)
   __nv_bfloat16 *dk_out, *dv_out;  // mode-0 items when causal_fp32 == 0: [kv tokens, h_kv, D] bf16
   float *dk_acc, *dv_acc;   // fp32 [prompt tokens, h_kv, D]: mode-1 items, and mode-0 items when causal_fp32 != 0
   long long n_tiles;        // query tiles in the stats table
@@ -43,6 +43,10 @@ struct BwdParams {
 };
 
 constexpr int kBwdThreads = 576;  // 16 element-wise warps, TMA warp, MMA warp
+#ifndef AUGTREE_BWD_FMA_MASK
+#define AUGTREE_BWD_FMA_MASK 0x8888u
+#endif
+constexpr uint32_t kBwdFmaMask = AUGTREE_BWD_FMA_MASK;  // pairs (of a thread's 16) whose exp2 runs on the FMA pipe
 
 template <int D>
 struct BwdSmem {
@@ -270,13 +274,17 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       uint32_t sv[32];
       tmem_ld32(tR0 + lane_off + ch * 32, sv);
       tc_wait_ld();
+      // packed fp32: one fma per pair for the scale-and-subtract (the table holds -lse*log2e), and the pairs
+      // that kBwdFmaMask names take their exp2 on the FMA pipe
+      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
 #pragma unroll
       for (int i = 0; i < 32; i += 4) {
         const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + i);
-        pr[i + 0] = ex2(fmaf(__uint_as_float(sv[i + 0]), p.scale_log2, -l4.x));
-        pr[i + 1] = ex2(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -l4.y));
-        pr[i + 2] = ex2(fmaf(__uint_as_float(sv[i + 2]), p.scale_log2, -l4.z));
-        pr[i + 3] = ex2_fma(fmaf(__uint_as_float(sv[i + 3]), p.scale_log2, -l4.w));  // one in four on the FMA pipe
+        const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(sv[i + 0]), __uint_as_float(sv[i + 1])), sc2, make_float2(l4.x, l4.y));
+        const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])), sc2, make_float2(l4.z, l4.w));
+        const float2 p0 = ((kBwdFmaMask >> (i / 2)) & 1) ? ex2_fma2(x0) : ex2_2(x0);
+        const float2 p1 = ((kBwdFmaMask >> (i / 2 + 1)) & 1) ? ex2_fma2(x1) : ex2_2(x1);
+        pr[i + 0] = p0.x; pr[i + 1] = p0.y; pr[i + 2] = p1.x; pr[i + 3] = p1.y;
       }
       if (!all_visible) {
 #pragma unroll
@@ -322,15 +330,16 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               tmem_ld32(tR1 + lane_off + ch * 32, dpv);
               tc_wait_ld();
               uint32_t dd[16];
+              const float2 sc2 = make_float2(p.scale, p.scale);
 #pragma unroll
               for (int i = 0; i < 32; i += 4) {
-                const float4 d4 = *reinterpret_cast<const float4 *>(dl + i);
-                const float a0 = pr[i + 0] * fmaf(__uint_as_float(dpv[i + 0]), p.scale, -d4.x);
-                const float a1 = pr[i + 1] * fmaf(__uint_as_float(dpv[i + 1]), p.scale, -d4.y);
-                const float a2 = pr[i + 2] * fmaf(__uint_as_float(dpv[i + 2]), p.scale, -d4.z);
-                const float a3 = pr[i + 3] * fmaf(__uint_as_float(dpv[i + 3]), p.scale, -d4.w);
-                dd[i / 2] = pack_bf16(a0, a1);
-                dd[i / 2 + 1] = pack_bf16(a2, a3);
+                const float4 d4 = *reinterpret_cast<const float4 *>(dl + i);   // -scale * delta
+                const float2 t0 = __ffma2_rn(make_float2(__uint_as_float(dpv[i + 0]), __uint_as_float(dpv[i + 1])), sc2, make_float2(d4.x, d4.y));
+                const float2 t1 = __ffma2_rn(make_float2(__uint_as_float(dpv[i + 2]), __uint_as_float(dpv[i + 3])), sc2, make_float2(d4.z, d4.w));
+                const float2 a0 = __fmul2_rn(make_float2(pr[i + 0], pr[i + 1]), t0);
+                const float2 a1 = __fmul2_rn(make_float2(pr[i + 2], pr[i + 3]), t1);
+                dd[i / 2] = pack_bf16(a0.x, a0.y);
+                dd[i / 2 + 1] = pack_bf16(a1.x, a1.y);
               }
               tmem_st16(tR1 + lane_off + ch * 32, dd);
             }
@@ -404,9 +413,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   if (warp == 17) { tc_fence_after(); tmem_dealloc(tmem, 512); }
 }
 
-// Row statistics of the backward pass, stored per 128-row query tile:
-// stats[head][tile][0][i] = lse * log2(e) (+inf for rows past the tile's end),
-// stats[head][tile][1][i] = scale * sum_d dO * O (0 past the end).  One warp per 16 rows.
+// Row statistics of the backward pass, stored per 128-row query tile, negated so that the tile kernels
+// fold them in with one fused multiply-add:
+// stats[head][tile][0][i] = -lse * log2(e) (-inf for rows past the tile's end: their P becomes 0),
+// stats[head][tile][1][i] = -scale * sum_d dO * O (0 past the end).  One warp per 16 rows.
 template <int D>
 __global__ void bwd_preprocess_kernel(const __nv_bfloat16 *o, const __nv_bfloat16 *d_o, const float *lse, const int32_t *tiles,
                                       float *stats, long long n_tok, long long n_tiles, int h_q, float scale) {
@@ -414,19 +424,39 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16 *o, const __nv_bfloat1
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tok0 = tiles[2 * tile], rows = tiles[2 * tile + 1];
   float *out = stats + ((long long)head * n_tiles + tile) * 256;
-  constexpr int PER = D / 32;
-  for (int i = warp; i < 128; i += 8) {
-    float acc = 0.f, l2 = INFINITY;
+  // a lane reads 16 bytes of a row: D / 8 lanes per row, 32 / (D / 8) rows per warp pass; a warp owns 16 rows and
+  // issues the loads of all its passes before it reduces any (HBM-bound: keep many loads in flight)
+  constexpr int LPR = D / 8, RPP = 32 / LPR, PASSES = 16 / RPP;
+  const int sub = lane / LPR, part = lane % LPR;
+  uint4 vo[PASSES], vd[PASSES];
+#pragma unroll
+  for (int ps = 0; ps < PASSES; ++ps) {
+    const int i = warp * 16 + ps * RPP + sub;
+    vo[ps] = make_uint4(0, 0, 0, 0); vd[ps] = make_uint4(0, 0, 0, 0);
     if (i < rows) {
-      const long long w = ((long long)tok0 + i) * h_q + head;
-      const __nv_bfloat16 *po = o + w * D + lane * PER, *pd = d_o + w * D + lane * PER;
-#pragma unroll
-      for (int e = 0; e < PER; ++e) acc += __bfloat162float(po[e]) * __bfloat162float(pd[e]);
-#pragma unroll
-      for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-      l2 = lse[(long long)head * n_tok + tok0 + i] * 1.4426950408889634f;
+      const long long w = (((long long)tok0 + i) * h_q + head) * D + part * 8;
+      vo[ps] = *reinterpret_cast<const uint4 *>(o + w);
+      vd[ps] = *reinterpret_cast<const uint4 *>(d_o + w);
     }
-    if (lane == 0) { out[i] = l2; out[128 + i] = acc * scale; }
+  }
+#pragma unroll
+  for (int ps = 0; ps < PASSES; ++ps) {
+    const int i = warp * 16 + ps * RPP + sub;
+    const uint32_t a[4] = {vo[ps].x, vo[ps].y, vo[ps].z, vo[ps].w}, b[4] = {vd[ps].x, vd[ps].y, vd[ps].z, vd[ps].w};
+    float acc = 0.f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&a[e]));
+      const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&b[e]));
+      acc = fmaf(x.x, y.x, fmaf(x.y, y.y, acc));
+    }
+#pragma unroll
+    for (int sft = LPR / 2; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+    if (part == 0) {
+      const bool valid = i < rows;
+      out[i] = valid ? -lse[(long long)head * n_tok + tok0 + i] * 1.4426950408889634f : -INFINITY;
+      out[128 + i] = valid ? -acc * scale : 0.f;
+    }
   }
 }
 

@@ -27,7 +27,7 @@ struct DqParams {
   const int32_t *items;     // lane order, 12 ints: q_tok0, q_pos0, q_rows, head, a_tok0, a_len, b_tok0, b_len,
                             //                      stats tile index, 1, weight, kv head
   const int32_t *lane_ptr;  // [gridDim.x + 1]
-  const float *stats;       // [h_q][n_tiles][2][128]: lse*log2e (inf past the end), scale*rowsum(dO*O)
+  const float *stats;       // [h_q][n_tiles][2][128]: -lse*log2e (-inf past the end), -scale*rowsum(dO*O)
   __nv_bfloat16 *dq;        // [query tokens, h_q, D]
   long long n_tiles;
   int h_q;
@@ -36,6 +36,10 @@ struct DqParams {
 };
 
 constexpr int kDqThreads = 320;
+#ifndef AUGTREE_DQ_FMA_MASK
+#define AUGTREE_DQ_FMA_MASK 0x8888u
+#endif
+constexpr uint32_t kDqFmaMask = AUGTREE_DQ_FMA_MASK;  // pairs (period 16) whose exp2 runs on the FMA pipe
 
 template <int D>
 struct DqSmem {
@@ -225,8 +229,8 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       // ---- Q and dO rows into TMEM as bf16 A operands; this thread: row r, columns (D/2)*ch .. of d
       ok = mbar_wait(bar_qdo_full, ic & 1, ab, WAIT_DQ_QDO);
       if (!ok) break;
-      const float lse2 = reinterpret_cast<const float *>(smem_raw + SM::kOffStats)[r];
-      const float dlt = reinterpret_cast<const float *>(smem_raw + SM::kOffStats)[128 + r];
+      const float nlse2 = reinterpret_cast<const float *>(smem_raw + SM::kOffStats)[r];        // -lse * log2(e)
+      const float ndlt = reinterpret_cast<const float *>(smem_raw + SM::kOffStats)[128 + r];   // -scale * delta
       {
         constexpr int NCH = D / 16;  // 16-byte chunks per thread (8 for D=128: one whole box; 4 for D=64: half a box)
         const int box = (D == 128) ? ch : 0, c0 = (D == 128) ? 0 : ch * 4;
@@ -264,10 +268,13 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           // number of leading key columns of this tile that the row sees
           const int limit = (i < nA) ? (a_len - i * 128) : (q_pos0 + r + 1 - (i - nA) * 128);
           const int lim = limit - ch * 64;
+          // packed fp32 for the scale-and-subtract; the pairs kDqFmaMask names take exp2 on the FMA pipe
+          const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nl2 = make_float2(nlse2, nlse2);
 #pragma unroll
-          for (int c = 0; c < 64; ++c) {  // one exponential in four on the FMA pipe, the rest on the special-function unit
-            const float x = fmaf(__uint_as_float(sv[c]), p.scale_log2, -lse2);
-            pr[c] = (c & 3) == 3 ? ex2_fma(x) : ex2(x);
+          for (int c = 0; c < 64; c += 2) {
+            const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), sc2, nl2);
+            const float2 e = ((kDqFmaMask >> ((c / 2) & 15)) & 1) ? ex2_fma2(x) : ex2_2(x);
+            pr[c] = e.x; pr[c + 1] = e.y;
           }
           if (lim < 64) {
 #pragma unroll
@@ -280,6 +287,7 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         if (!ok) break;
         tc_fence_after();
         {
+          const float2 sc2 = make_float2(p.scale, p.scale), nd2 = make_float2(ndlt, ndlt);
           uint32_t dpv[64];
           tmem_ld32(tDP + lane_off + ch * 64, *reinterpret_cast<uint32_t(*)[32]>(&dpv[0]));
           tmem_ld32(tDP + lane_off + ch * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&dpv[32]));
@@ -289,9 +297,9 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             uint32_t dd[16];
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-              const float a0 = pr[c * 32 + 2 * e] * fmaf(__uint_as_float(dpv[c * 32 + 2 * e]), p.scale, -dlt);
-              const float a1 = pr[c * 32 + 2 * e + 1] * fmaf(__uint_as_float(dpv[c * 32 + 2 * e + 1]), p.scale, -dlt);
-              dd[e] = pack_bf16(a0, a1);
+              const float2 t = __ffma2_rn(make_float2(__uint_as_float(dpv[c * 32 + 2 * e]), __uint_as_float(dpv[c * 32 + 2 * e + 1])), sc2, nd2);
+              const float2 a = __fmul2_rn(make_float2(pr[c * 32 + 2 * e], pr[c * 32 + 2 * e + 1]), t);
+              dd[e] = pack_bf16(a.x, a.y);
             }
             tmem_st16(tDP + lane_off + ch * 64 + c * 16, dd);
           }

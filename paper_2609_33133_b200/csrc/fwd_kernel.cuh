@@ -32,11 +32,33 @@ struct FwdParams {
   long long n_tok;          // tokens in the query tensor
   int h_q;
   float scale_log2;         // softmax scale * log2(e)
+  const float *kmax2;       // [h_kv] largest squared key norm of the call's K tensors (key_norm_kernel)
   int *status;
 };
 
 constexpr int kFwdThreads = 320;
-constexpr float kRescaleThreshold = 8.0f;  // log2 units: P stays <= 2^8
+constexpr float kRescaleThreshold = 8.0f;  // log2 units: P stays <= 2^8 while the row maximum is tracked
+// When |q_a| max_b |k_b| scale log2(e) (a bound on every score of row a, by Cauchy-Schwarz) is less than this many
+// log2 units above the row's maximum over its first KV tile, no later exponential can exceed 2^60: with fp32
+// accumulators and bf16's fp32-sized exponent nothing overflows and nothing loses precision (softmax does not
+// depend on the reference), so the row maximum of the later tiles is not computed at all.
+constexpr float kSkipMaxHeadroom = 60.0f;
+#ifndef AUGTREE_FWD_SPLIT_WG
+#define AUGTREE_FWD_SPLIT_WG 0
+#endif
+#ifndef AUGTREE_FWD_FMA_MASK
+#define AUGTREE_FWD_FMA_MASK 0x8888u
+#endif
+constexpr uint32_t kFwdFmaMask = AUGTREE_FWD_FMA_MASK;  // column blocks (of 16) whose exp2 runs on the FMA pipe
+
+#if AUGTREE_TRACE
+// Measurement build only: clock64 spans of the softmax phases, summed over warp 1 of every CTA
+// (0 wait for S, 1 TMEM load, 6 maxima, 7 quad shuffles, 2 rescale test, 3 exponentials, 4 store + hand-off; 5 = passes).
+__device__ unsigned long long g_fwd_trace[8];
+#define TRACE_MARK(k) do { const long long t_ = clock64(); tr[k] += t_ - t_prev; t_prev = t_; } while (0)
+#else
+#define TRACE_MARK(k) do { } while (0)
+#endif
 
 template <int D>
 struct FwdSmem {
@@ -74,7 +96,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    mbar_init(bar_q_full, 1); mbar_init(bar_q_empty, 1);
+    mbar_init(bar_q_full, 1); mbar_init(bar_q_empty, 1 + 8);  // Q slot free: last S MMA of the item done, 8 warps read their rows
     for (int s = 0; s < NS; ++s) { mbar_init(bar_kv_full + 8 * s, 1); mbar_init(bar_kv_empty + 8 * s, 1); }
     for (int g = 0; g < 2; ++g) {
       mbar_init(bar_s_full + 8 * g, 1); mbar_init(bar_p_full + 8 * g, 8);
@@ -256,10 +278,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // accumulator-fragment layout (16x256b): thread t holds rows t/4 and t/4 + 8, and of every block of 8
     // columns the two columns 2 (t % 4), 2 (t % 4) + 1.  A row lives in one quad, so its maximum and sum are
     // two shuffles and no warp waits for another.
-    const int lane_base = (warp & 3) * 32 + (warp >> 2) * 16;
-    const int rA = lane_base + (lane >> 2), rB = rA + 8;   // rows inside the query tile
     const int cq = 2 * (lane & 3);                         // first of this thread's two columns in a block of 8
-    const uint32_t lane_off = (uint32_t)lane_base << 16;
+#if AUGTREE_FWD_SPLIT_WG
+    // warps 0-3 own query tile 0, warps 4-7 query tile 1; a warp does its 32 rows as two blocks of 16 (u = 0, 1)
+#define FWD_UNIT(u) const int g = warp >> 2, lane_base = (warp & 3) * 32 + (u) * 16
+#else
+    // all eight warps work on query tile u = 0, then on tile 1; a warp does 16 rows of each
+#define FWD_UNIT(u) const int g = (u), lane_base = (warp & 3) * 32 + (warp >> 2) * 16
+#endif
     auto quad_max = [](float x) {
       x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 1));
       return fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 2));
@@ -270,23 +296,71 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     };
     uint32_t ic = 0, T = 0;
     bool ok = true;
+#if AUGTREE_TRACE
+    long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0}, t_prev = clock64();
+#endif
     for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
       const int32_t *I = p.items + (size_t)it * 12;
       const int q_tok0 = I[0], q_pos0 = I[1], q_rows = I[2], head = I[3], a_len = I[5], b_len = I[7];
       const int split = I[8], n_splits = I[9];
       const int nA = (a_len + 127) >> 7, n = nA + ((b_len + 127) >> 7);
-      // per tile g and row (A, B): running reference maximum and this thread's share of the row sum
+      // per unit u and row (A, B): running reference maximum and this thread's share of the row sum
       float mA[2] = {0.f, 0.f}, mB[2] = {0.f, 0.f}, lA[2] = {0.f, 0.f}, lB[2] = {0.f, 0.f};
+      // upper bounds of the rows' scores (log2 units) from the query rows in shared memory and the largest key norm;
+      // skip[u]: the warp's rows of unit u have enough headroom to leave the reference maximum where tile 0 put it
+      float bndA[2], bndB[2];
+      bool skip[2] = {false, false};
+      ok = mbar_wait(bar_q_full, ic & 1, ab, WAIT_FWD_Q_FULL);
+      if (!ok) break;
+      {
+        const float kscale = sqrtf(p.kmax2[I[11]]) * p.scale_log2 * 1.0001f;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          FWD_UNIT(u);
+          const int rA = lane_base + (lane >> 2), rB = rA + 8;
+          float nA2 = 0.f, nB2 = 0.f;
+          // a row is NBOX lines of 128 bytes (8 chunks of 16, swizzled among themselves): each thread of the quad
+          // squares two chunks of every line, whichever elements they hold
+#pragma unroll
+          for (int b = 0; b < NBOX; ++b)
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+              const uint4 xa = *reinterpret_cast<const uint4 *>(smem_raw + SM::kOffQ + g * TILE + b * 16384 + rA * 128 + (((lane & 3) + 4 * c) << 4));
+              const uint4 xb = *reinterpret_cast<const uint4 *>(smem_raw + SM::kOffQ + g * TILE + b * 16384 + rB * 128 + (((lane & 3) + 4 * c) << 4));
+              const uint32_t wa[4] = {xa.x, xa.y, xa.z, xa.w}, wb[4] = {xb.x, xb.y, xb.z, xb.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&wa[e]));
+                const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&wb[e]));
+                nA2 = fmaf(fa.x, fa.x, fmaf(fa.y, fa.y, nA2));
+                nB2 = fmaf(fb.x, fb.x, fmaf(fb.y, fb.y, nB2));
+              }
+            }
+          bndA[u] = sqrtf(quad_sum(nA2)) * kscale;
+          bndB[u] = sqrtf(quad_sum(nB2)) * kscale;
+        }
+      }
+      // the query tiles may be overwritten by the next item's only after every softmax warp has read its rows
+      // (this also keeps the softmax warps within one phase of bar_q_full: the next load cannot complete before)
+      warp_arrive(bar_q_empty);
       for (int j = 0; j < n && ok; ++j, ++T) {
 #pragma unroll
-        for (int g = 0; g < 2; ++g) {
+        for (int u = 0; u < 2; ++u) {
+          FWD_UNIT(u);
+          const int rA = lane_base + (lane >> 2), rB = rA + 8;   // rows inside the query tile
+          const uint32_t lane_off = (uint32_t)lane_base << 16;
           const uint32_t tS = tmem + lane_off + g * 128, tO = tmem + lane_off + 256 + g * 128;
+#if AUGTREE_TRACE
+          t_prev = clock64();
+#endif
           ok = mbar_wait(bar_s_full + 8 * g, T & 1, ab, WAIT_FWD_S_FULL);
           if (!ok) break;
           tc_fence_after();
+          TRACE_MARK(0);
           uint32_t s[64];
           tmem_ld_16x256b_x16(tS, s);
           tc_wait_ld();
+          TRACE_MARK(1);
           // number of leading key columns of this KV tile that rows A and B see
           const int lim0 = (j < nA) ? (a_len - j * 128) : (q_pos0 + g * 128 + 1 - (j - nA) * 128);
           const int limA = (j < nA) ? lim0 : lim0 + rA, limB = (j < nA) ? lim0 : lim0 + rB;
@@ -300,76 +374,98 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               if (c + 1 >= limB) s[4 * i + 3] = 0xff800000u;
             }
           }
-          // row maxima of the raw scores (the scale is positive, so it commutes with the maximum)
-          float xA = -INFINITY, xB = -INFINITY;
+          if (!skip[u]) {
+            // row maxima of the raw scores (the scale is positive, so it commutes with the maximum)
+            float xA, xB;
+            {
+              float a0 = -INFINITY, a1 = -INFINITY, b0 = -INFINITY, b1 = -INFINITY;   // two chains per row: shorter dependency
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            xA = max3(xA, __uint_as_float(s[4 * i]), __uint_as_float(s[4 * i + 1]));
-            xB = max3(xB, __uint_as_float(s[4 * i + 2]), __uint_as_float(s[4 * i + 3]));
-          }
-          xA = quad_max(xA) * p.scale_log2;
-          xB = quad_max(xB) * p.scale_log2;
-          if (j == 0) {
-            mA[g] = (xA == -INFINITY) ? 0.f : xA;
-            mB[g] = (xB == -INFINITY) ? 0.f : xB;
-          } else {
-            const bool needA = xA > mA[g] + kRescaleThreshold, needB = xB > mB[g] + kRescaleThreshold;
-            if (__any_sync(0xffffffffu, needA || needB)) {
-              ok = mbar_wait(bar_o_full + 8 * g, (T - 1) & 1, ab, WAIT_FWD_O_FULL);  // PV_g(j-1) done
-              if (!ok) break;
-              tc_fence_after();
-              float alA = 1.f, alB = 1.f;
-              if (needA) { alA = ex2(mA[g] - xA); mA[g] = xA; lA[g] *= alA; }
-              if (needB) { alB = ex2(mB[g] - xB); mB[g] = xB; lB[g] *= alB; }
+              for (int i = 0; i < 16; i += 2) {
+                a0 = max3(a0, __uint_as_float(s[4 * i]), __uint_as_float(s[4 * i + 1]));
+                b0 = max3(b0, __uint_as_float(s[4 * i + 2]), __uint_as_float(s[4 * i + 3]));
+                a1 = max3(a1, __uint_as_float(s[4 * i + 4]), __uint_as_float(s[4 * i + 5]));
+                b1 = max3(b1, __uint_as_float(s[4 * i + 6]), __uint_as_float(s[4 * i + 7]));
+              }
+              xA = fmaxf(a0, a1);
+              xB = fmaxf(b0, b1);
+            }
+            TRACE_MARK(6);
+            xA = quad_max(xA) * p.scale_log2;
+            xB = quad_max(xB) * p.scale_log2;
+            TRACE_MARK(7);
+            if (j == 0) {
+              mA[u] = (xA == -INFINITY) ? 0.f : xA;
+              mB[u] = (xB == -INFINITY) ? 0.f : xB;
+              skip[u] = __all_sync(0xffffffffu, bndA[u] - mA[u] < kSkipMaxHeadroom && bndB[u] - mB[u] < kSkipMaxHeadroom);
+            } else {
+              const bool needA = xA > mA[u] + kRescaleThreshold, needB = xB > mB[u] + kRescaleThreshold;
+              if (__any_sync(0xffffffffu, needA || needB)) {
+                ok = mbar_wait(bar_o_full + 8 * g, (T - 1) & 1, ab, WAIT_FWD_O_FULL);  // PV_g(j-1) done
+                if (!ok) break;
+                tc_fence_after();
+                float alA = 1.f, alB = 1.f;
+                if (needA) { alA = ex2(mA[u] - xA); mA[u] = xA; lA[u] *= alA; }
+                if (needB) { alB = ex2(mB[u] - xB); mB[u] = xB; lB[u] *= alB; }
 #pragma unroll 1
-              for (int c = 0; c < D / 32; ++c) {
-                uint32_t o[16];
-                tmem_ld_16x256b_x4(tO + c * 32, o);
-                tc_wait_ld();
+                for (int c = 0; c < D / 32; ++c) {
+                  uint32_t o[16];
+                  tmem_ld_16x256b_x4(tO + c * 32, o);
+                  tc_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  o[4 * i] = __float_as_uint(__uint_as_float(o[4 * i]) * alA);
-                  o[4 * i + 1] = __float_as_uint(__uint_as_float(o[4 * i + 1]) * alA);
-                  o[4 * i + 2] = __float_as_uint(__uint_as_float(o[4 * i + 2]) * alB);
-                  o[4 * i + 3] = __float_as_uint(__uint_as_float(o[4 * i + 3]) * alB);
+                  for (int i = 0; i < 4; ++i) {
+                    o[4 * i] = __float_as_uint(__uint_as_float(o[4 * i]) * alA);
+                    o[4 * i + 1] = __float_as_uint(__uint_as_float(o[4 * i + 1]) * alA);
+                    o[4 * i + 2] = __float_as_uint(__uint_as_float(o[4 * i + 2]) * alB);
+                    o[4 * i + 3] = __float_as_uint(__uint_as_float(o[4 * i + 3]) * alB);
+                  }
+                  tmem_st_16x256b_x4(tO + c * 32, o);
                 }
-                tmem_st_16x256b_x4(tO + c * 32, o);
               }
             }
           }
-          // P = exp2(s * scale - m), bf16 pairs in the 16x128b layout over the S columns [0, 64).  One block of
-          // columns in four takes its exponentials on the FMA pipe, the rest on the special-function unit.
-          float sA = 0.f, sB = 0.f;
-          const float ma = mA[g], mb = mB[g];
+          TRACE_MARK(2);
+          // P = exp2(s * scale - m), bf16 pairs in the 16x128b layout over the S columns [0, 64).  The scale-and-
+          // subtract, the row sums and the polynomial exponentials run on register pairs (packed fp32: half the
+          // issue slots); kFwdFmaMask says which of the 16 column blocks take their exponentials on the FMA
+          // pipe instead of the special-function unit.
+          const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+          const float2 nmA = make_float2(-mA[u], -mA[u]), nmB = make_float2(-mB[u], -mB[u]);
+          float2 accA = make_float2(0.f, 0.f), accB = make_float2(0.f, 0.f);
           uint32_t pk[32];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float x0 = fmaf(__uint_as_float(s[4 * i]), p.scale_log2, -ma);
-            const float x1 = fmaf(__uint_as_float(s[4 * i + 1]), p.scale_log2, -ma);
-            const float x2 = fmaf(__uint_as_float(s[4 * i + 2]), p.scale_log2, -mb);
-            const float x3 = fmaf(__uint_as_float(s[4 * i + 3]), p.scale_log2, -mb);
-            float p0, p1, p2, p3;
-            if ((i & 3) == 3) { p0 = ex2_fma(x0); p1 = ex2_fma(x1); p2 = ex2_fma(x2); p3 = ex2_fma(x3); }
-            else { p0 = ex2(x0); p1 = ex2(x1); p2 = ex2(x2); p3 = ex2(x3); }
-            sA += p0 + p1;
-            sB += p2 + p3;
-            pk[2 * i] = pack_bf16(p0, p1);
-            pk[2 * i + 1] = pack_bf16(p2, p3);
+            const float2 xa = __ffma2_rn(make_float2(__uint_as_float(s[4 * i]), __uint_as_float(s[4 * i + 1])), sc2, nmA);
+            const float2 xb = __ffma2_rn(make_float2(__uint_as_float(s[4 * i + 2]), __uint_as_float(s[4 * i + 3])), sc2, nmB);
+            float2 pa, pb;
+            if ((kFwdFmaMask >> i) & 1) { pa = ex2_fma2(xa); pb = ex2_fma2(xb); }
+            else { pa = ex2_2(xa); pb = ex2_2(xb); }
+            accA = __fadd2_rn(accA, pa);
+            accB = __fadd2_rn(accB, pb);
+            pk[2 * i] = pack_bf16(pa.x, pa.y);
+            pk[2 * i + 1] = pack_bf16(pb.x, pb.y);
           }
+          const float sA = accA.x + accA.y, sB = accB.x + accB.y;
+          TRACE_MARK(3);
           tmem_st_16x128b_x16(tS, pk);
-          lA[g] += sA;
-          lB[g] += sB;
+          lA[u] += sA;
+          lB[u] += sB;
           tc_wait_st();
           tc_fence_before();
           warp_arrive(bar_p_full + 8 * g);
+          TRACE_MARK(4);
+#if AUGTREE_TRACE
+          ++tr[5];
+#endif
         }
       }
       if (!ok) break;
       // ---- epilogue: O / l, LSE = ln2 * (m + log2 l); a thread writes two columns of each block of 8 of its rows
 #pragma unroll
-      for (int g = 0; g < 2; ++g) {
-        const uint32_t tO = tmem + lane_off + 256 + g * 128;
-        const float ltA = quad_sum(lA[g]), ltB = quad_sum(lB[g]);
+      for (int u = 0; u < 2; ++u) {
+        FWD_UNIT(u);
+        const int rA = lane_base + (lane >> 2), rB = rA + 8;
+        const uint32_t tO = tmem + ((uint32_t)lane_base << 16) + 256 + g * 128;
+        const float ltA = quad_sum(lA[u]), ltB = quad_sum(lB[u]);
         ok = mbar_wait(bar_o_full + 8 * g, (T - 1) & 1, ab, WAIT_FWD_O_FULL);
         if (!ok) break;
         tc_fence_after();
@@ -398,7 +494,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           }
         }
         if ((lane & 3) == 0) {
-          const float lseA = (mA[g] + log2f(ltA)) * 0.6931471805599453f, lseB = (mB[g] + log2f(ltB)) * 0.6931471805599453f;
+          const float lseA = (mA[u] + log2f(ltA)) * 0.6931471805599453f, lseB = (mB[u] + log2f(ltB)) * 0.6931471805599453f;
           if (n_splits == 1) {
             if (validA) p.lse[(long long)head * p.n_tok + tokA] = lseA;
             if (validB) p.lse[(long long)head * p.n_tok + tokB] = lseB;
@@ -411,6 +507,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         warp_arrive(bar_o_empty + 8 * g);
       }
     }
+#if AUGTREE_TRACE
+    if (warp == 1 && lane == 0)
+      for (int k = 0; k < 8; ++k) atomicAdd(&g_fwd_trace[k], (unsigned long long)tr[k]);
+#endif
   }
 
   // ---------------------------------------------------------------- teardown
@@ -424,6 +524,43 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   tc_fence_before();
   __syncthreads();
   if (warp == 9) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+}
+
+// Largest squared key norm per KV head over the K tensors of one forward call (the unmasked-range tensor and,
+// if different, the causal-range tensor): out[h] = max over tokens of |k[token, h, :]|^2, as the bits of a
+// non-negative float (so an unsigned atomicMax orders them).  `out` is cleared by the caller before the launch.
+// Feeds the score bound that lets the tile kernel skip row maxima; HBM-bound, a few microseconds.
+template <int D>
+__global__ void key_norm_kernel(const __nv_bfloat16 *ka, long long a_tok, const __nv_bfloat16 *kb, long long b_tok, int h_kv,
+                                unsigned int *out) {
+  constexpr int LPR = D / 8, RPP = 32 / LPR;   // 16-byte loads: lanes per (token, head) row, rows per warp pass
+  const int lane = threadIdx.x & 31, sub = lane / LPR, part = lane % LPR;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5, n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const int head = blockIdx.y;
+  float best = 0.f;
+  for (int which = 0; which < 2; ++which) {
+    const __nv_bfloat16 *k = which ? kb : ka;
+    const long long n = which ? b_tok : a_tok;
+    for (long long t0 = warp * RPP; t0 < n; t0 += n_warps * RPP) {
+      const long long t = t0 + sub;
+      float acc = 0.f;
+      if (t < n) {
+        const uint4 x = *reinterpret_cast<const uint4 *>(k + (t * h_kv + head) * D + part * 8);
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&w[e]));
+          acc = fmaf(f.x, f.x, fmaf(f.y, f.y, acc));
+        }
+      }
+#pragma unroll
+      for (int sft = LPR / 2; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+      best = fmaxf(best, acc);
+    }
+  }
+#pragma unroll
+  for (int sft = 16; sft > 0; sft >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, sft));
+  if (lane == 0) atomicMax(out + head, __float_as_uint(best));
 }
 
 // Merge of the prompt-KV shards' partial states (Sec. 3.3): one warp per

@@ -74,7 +74,7 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
   p->flags = d->flags;
   p->n_lanes = d->n_lanes;
   p->kv_splits = d->kv_splits < 1 ? 1 : d->kv_splits;
-  if (p->kv_splits > 64) return AUGTREE_ERR_UNSUPPORTED;
+  if (p->kv_splits > 64 || p->h_kv > 64) return AUGTREE_ERR_UNSUPPORTED;
 
   p->prompt_len.assign(d->prompt_len, d->prompt_len + d->n_groups);
   p->n_br.assign(d->n_branches, d->n_branches + d->n_groups);
@@ -226,9 +226,10 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
   // scratch sizes (bytes, each region 256-byte aligned)
   auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
   const size_t hq = (size_t)p->h_q, dd = (size_t)p->head_dim;
-  p->ws_fwd = 0;
+  // forward: 256 bytes for the per-KV-head key-norm maxima, then (with prompt-KV shards) the shards' partial states
+  p->ws_fwd = 256;
   if (p->max_splits > 1)
-    p->ws_fwd = al((size_t)p->max_splits * (size_t)tr * hq * dd * 4) + al((size_t)p->max_splits * (size_t)tr * hq * 4);
+    p->ws_fwd += al((size_t)p->max_splits * (size_t)tr * hq * dd * 4) + al((size_t)p->max_splits * (size_t)tr * hq * 4);
   const size_t tmax = (size_t)std::max<int64_t>(tp, tr);
   // backward: row statistics [H_q][tiles][2][128] fp32
   const size_t ntile = std::max(p->tiles_replay.size(), p->tiles_prefill.size()) / 2;

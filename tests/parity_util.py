@@ -138,9 +138,11 @@ def rounding_error_sigma(w, t_cpu, bf16_prompt_grads=False):
     return {name: np.sqrt(x) for name, x in var.items()}
 
 
-def assert_parity_elementwise(got, ref, sigma):
+def assert_parity_elementwise(got, ref, sigma, rel_l2=None):
     """rel-L2 <= 5e-3 per tensor and |LSE error| <= 1e-3 as stated; the absolute error of every element
-    <= max(2e-2, SIGMAS x its modelled rounding-error standard deviation)."""
+    <= max(2e-2, SIGMAS x its modelled rounding-error standard deviation).  `rel_l2`: {tensor: bound} for a
+    named case whose test states why."""
+    rel_l2 = rel_l2 or {}
     rows = errors(got, ref)
     bad = []
     for k, (rel, mx, finite) in rows.items():
@@ -152,7 +154,7 @@ def assert_parity_elementwise(got, ref, sigma):
         else:
             bound = np.maximum(MAX_ABS, SIGMAS * sigma[k])
             over = np.abs(got[k] - ref[k]) - bound
-            if rel > REL_L2 or over.max() > 0:
+            if rel > rel_l2.get(k, REL_L2) or over.max() > 0:
                 i = np.unravel_index(int(np.argmax(over)), over.shape)
                 bad.append((k, rel, mx, "worst element", i, float(np.abs(got[k] - ref[k])[i]), "bound", float(bound[i])))
     assert not bad, f"parity failures: {bad}; all: {rows}"

@@ -30,11 +30,16 @@ def test_autograd_wrapper_matches_oracle():
     f64 = lambda v: v.detach().float().cpu().numpy().astype(np.float64)
     got = {"o_p": f64(o_p), "o_r": f64(o_r), "dq_p": f64(x["q_p"].grad), "dk_p": f64(x["k_p"].grad), "dv_p": f64(x["v_p"].grad),
            "dq_r": f64(x["q_r"].grad), "dk_r": f64(x["k_r"].grad), "dv_r": f64(x["v_r"].grad)}
-    # the prompt-KV gradients as accumulated (fp32): the stated bounds, flat
+    ref = {k: ref[k] for k in got}
+    sigma = pu.rounding_error_sigma(w, t, bf16_prompt_grads=True)
+    # as autograd delivers them (every gradient in bf16, like its input): relative L2 as stated; element-wise
+    # max(2e-2, six sigma of the modelled rounding error, delivery included), because a bf16 value of magnitude
+    # 4-8 is rounded by up to 1.6e-2 on delivery alone and the first rows of a prompt carry large dS roundings
+    # (measured here: one element of dq_p, |ref| = 6.6, off by 2.4e-2)
+    pu.assert_parity_elementwise(got, ref, sigma)
+    # the outputs and the prompt-KV gradients as accumulated (fp32): the stated bounds, flat
     acc = {"dk_p": f64(plan.prompt_grad_fp32[0]), "dv_p": f64(plan.prompt_grad_fp32[1])}
-    pu.assert_parity({**got, **acc}, {k: ref[k] for k in got})
-    # ... and as autograd delivers them, in bf16 like their inputs: a value of magnitude 8-16 is rounded by up to
-    # 3.1e-2 on delivery alone, so the element-wise bound is max(2e-2, six sigma of the modelled rounding error, delivery included)
-    pu.assert_parity_elementwise(got, {k: ref[k] for k in got}, pu.rounding_error_sigma(w, t, bf16_prompt_grads=True))
+    flat = ("o_p", "o_r", "dk_p", "dv_p")
+    pu.assert_parity({**{k: got[k] for k in ("o_p", "o_r")}, **acc}, {k: ref[k] for k in flat})
     for k in ("dk_p", "dv_p"):   # the delivered copy is the accumulator rounded once
         assert np.array_equal(got[k], f64(torch.from_numpy(acc[k]).float().to(torch.bfloat16)))
