@@ -64,6 +64,23 @@ typedef enum {
 
 /* flags */
 #define AUGTREE_FLAG_ZERO_PROMPT_GRAD 1u /* replay_bwd clears dkp_acc/dvp_acc before accumulating */
+/*
+ * Fault injection for tests of the failure paths.  The faults are made on the
+ * host or by leaving work undone; none of them faults, traps or hangs the
+ * device, and a plan without these flags behaves as if they did not exist.
+ *  SHORT_WAIT     every device-side wait gives up after about a millisecond
+ *                 instead of about a second
+ *  SKIP_FWD_LOAD  lane 0 of the forward kernels never loads the first V tile of
+ *                 its first item: the wait for it runs out, the lane records
+ *                 AUGTREE_ERR_TIMEOUT and returns; the other lanes finish
+ *  SKIP_BWD_LOAD  the same for the first dO tile of the key-side backward kernel
+ *  DROP_ITEM      the device copy of the replay-forward lane table loses one
+ *                 item; augtree_items_completed then reports the shortfall
+ */
+#define AUGTREE_FLAG_TEST_SHORT_WAIT 0x100u
+#define AUGTREE_FLAG_TEST_SKIP_FWD_LOAD 0x200u
+#define AUGTREE_FLAG_TEST_SKIP_BWD_LOAD 0x400u
+#define AUGTREE_FLAG_TEST_DROP_ITEM 0x800u
 
 /*
  * Packed group descriptor (host, plain data).  One entry per replay tree
@@ -249,6 +266,17 @@ int augtree_replay_fwd_static(const augtree_plan_t *plan, const void *q_r, const
  * names the wait that gave up.  The word is cleared by the read.
  */
 int augtree_last_device_status(const augtree_plan_t *plan, int *status, int *detail);
+
+/*
+ * Work accounting (no counterpart in the paper's method).  Every tile kernel
+ * counts the work items it has finished; the host counts the items it has
+ * handed to launches.  Synchronises the plan's device and returns both counts
+ * for one kernel (numbering as in augtree_get_kernel_time), summed over the
+ * plan's lifetime.  completed < expected after a synchronised call means that
+ * some lane did not run or did not finish an item (a lane that gave up on a
+ * wait, a damaged lane table): its outputs are stale.
+ */
+int augtree_items_completed(const augtree_plan_t *plan, int kernel, long long *completed, long long *expected);
 
 /*
  * Measurement aid (no counterpart in the paper's method; Sec. 4.1 reports such

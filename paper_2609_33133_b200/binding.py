@@ -20,6 +20,7 @@ if not os.path.exists(LIB_PATH):
 lib = C.CDLL(LIB_PATH)
 
 FLAG_ZERO_PROMPT_GRAD = 1
+FLAG_TEST_SHORT_WAIT, FLAG_TEST_SKIP_FWD_LOAD, FLAG_TEST_SKIP_BWD_LOAD, FLAG_TEST_DROP_ITEM = 0x100, 0x200, 0x400, 0x800
 STATIC_SCRATCH_BYTES = 32 << 20
 FWD_ITEM_INTS, BWD_ITEM_INTS = 12, 8
 (TBL_CU_PROMPT, TBL_CU_BRANCH, TBL_CU_RESPONSE, TBL_PREFILL_FWD_ITEMS, TBL_PREFILL_FWD_LANE_PTR, TBL_PREFILL_FWD_ORDER,
@@ -31,7 +32,8 @@ FWD_ITEM_INTS, BWD_ITEM_INTS = 12, 8
 EXPORTS = ["augtree_plan_create", "augtree_plan_destroy", "augtree_plan_workspace_bytes", "augtree_plan_metadata",
            "augtree_prefill_fwd", "augtree_replay_fwd", "augtree_replay_bwd", "augtree_prefill_bwd",
            "augtree_last_device_status", "augtree_launch_count", "augtree_status_string",
-           "augtree_set_timing", "augtree_get_kernel_time", "augtree_replay_fwd_static", "augtree_assign_grid"]
+           "augtree_set_timing", "augtree_get_kernel_time", "augtree_replay_fwd_static", "augtree_assign_grid",
+           "augtree_items_completed"]
 
 
 class Desc(C.Structure):
@@ -55,6 +57,7 @@ lib.augtree_prefill_bwd.argtypes = [_vp] + [_vp] * 11 + [_vp, _sz, _vp]
 lib.augtree_last_device_status.argtypes = [_vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
 lib.augtree_set_timing.argtypes = [_vp, C.c_int]
 lib.augtree_get_kernel_time.argtypes = [_vp, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_int)]
+lib.augtree_items_completed.argtypes = [_vp, C.c_int, C.POINTER(C.c_longlong), C.POINTER(C.c_longlong)]
 lib.augtree_launch_count.restype = C.c_longlong
 lib.augtree_status_string.restype = C.c_char_p
 lib.augtree_status_string.argtypes = [C.c_int]
@@ -168,6 +171,12 @@ class Plan:
         ms, n = C.c_float(), C.c_int()
         _check(lib.augtree_get_kernel_time(self._h, kernel, C.byref(ms), C.byref(n)), "get_kernel_time")
         return ms.value, n.value
+
+    def items_completed(self, kernel: int):
+        """(items the kernel of schedule `kernel` has finished, items handed to its launches) over the plan's lifetime."""
+        done, want = C.c_longlong(), C.c_longlong()
+        _check(lib.augtree_items_completed(self._h, kernel, C.byref(done), C.byref(want)), "items_completed")
+        return done.value, want.value
 
     def device_status(self):
         s, d = C.c_int(), C.c_int()

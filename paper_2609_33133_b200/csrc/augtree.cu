@@ -75,17 +75,29 @@ int upload(const std::vector<int32_t> &h, int32_t **d) {
   return AUGTREE_OK;
 }
 
-int upload_sched(Sched &s, int n_lanes) {
+int upload_sched(Sched &s, int n_lanes, bool drop_last) {
   std::vector<int32_t> sorted(s.items.size());
   for (size_t i = 0; i < s.order.size(); ++i)
     std::memcpy(&sorted[i * s.item_ints], &s.items[(size_t)s.order[i] * s.item_ints], s.item_ints * sizeof(int32_t));
   int r = upload(sorted, &s.d_items);
   if (r) return r;
-  (void)n_lanes;
-  return upload(s.lane_ptr, &s.d_lane_ptr);
+  if (!drop_last) return upload(s.lane_ptr, &s.d_lane_ptr);
+  // injected fault (AUGTREE_FLAG_TEST_DROP_ITEM): the device copy of the lane table loses the last item of the
+  // last lane that has one; the host tables and the expected item count stay whole
+  std::vector<int32_t> lp = s.lane_ptr;
+  for (int l = n_lanes; l > 0; --l)
+    if (lp[l] > lp[l - 1]) {
+      for (int k = l; k <= n_lanes; ++k) --lp[k];
+      break;
+    }
+  return upload(lp, &s.d_lane_ptr);
 }
 
 void timing_mark(const augtree_plan *pl, int kind, bool stop, cudaStream_t st);
+
+long long wait_budget(const augtree_plan *pl) {
+  return (pl->flags & AUGTREE_FLAG_TEST_SHORT_WAIT) ? kWaitBudgetClocksTest : kWaitBudgetClocks;
+}
 
 template <int D>
 int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long q_tok, const void *ka, const void *va,
@@ -117,6 +129,9 @@ int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long 
   p.n_tok = q_tok; p.h_q = pl->h_q; p.scale_log2 = pl->scale * 1.4426950408889634f; p.status = pl->d_status;
   p.kmax2 = reinterpret_cast<const float *>(kmax2);
   const int kind = (int)(&s - pl->sched);
+  p.wait_budget = wait_budget(pl); p.kind = kind;
+  p.test_flags = (pl->flags & AUGTREE_FLAG_TEST_SKIP_FWD_LOAD) ? TEST_SKIP_FWD_LOAD : 0;
+  pl->launched_items[kind] += s.n_items();
   timing_mark(pl, kind, false, st);
   fwd_kernel<D><<<pl->n_lanes, kFwdThreads, FwdSmem<D>::kBytes, st>>>(mq, mka, mva, mkb, mvb, p);
   timing_mark(pl, kind, true, st);
@@ -168,6 +183,9 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     p.causal_fp32 = a.causal_fp32; p.scale = pl->scale; p.scale_log2 = pl->scale * 1.4426950408889634f;
     p.status = pl->d_status;
     const int kind = (int)(&s - pl->sched);
+    p.wait_budget = wait_budget(pl); p.kind = kind;
+    p.test_flags = (pl->flags & AUGTREE_FLAG_TEST_SKIP_BWD_LOAD) ? TEST_SKIP_BWD_LOAD : 0;
+    pl->launched_items[kind] += s.n_items();
     timing_mark(pl, kind, false, st);
     bwd_kernel<D><<<pl->n_lanes, kBwdThreads, BwdSmem<D>::kBytes, st>>>(mq, mdo, mk0, mv0, mk1, mv1, p);
     timing_mark(pl, kind, true, st);
@@ -183,6 +201,8 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     p.dq = static_cast<__nv_bfloat16 *>(a.dq); p.n_tiles = a.n_tiles; p.h_q = pl->h_q;
     p.scale = pl->scale; p.scale_log2 = pl->scale * 1.4426950408889634f; p.status = pl->d_status;
     const int kind = (int)(a.dq_sched - pl->sched);
+    p.wait_budget = wait_budget(pl); p.kind = kind;
+    pl->launched_items[kind] += a.dq_sched->n_items();
     timing_mark(pl, kind, false, st);
     // causal keys come from the queries' own sequence tensor (k0/v0)
     dq_kernel<D><<<pl->n_lanes, kDqThreads, DqSmem<D>::kBytes, st>>>(mq, mdo, mka, mva, mk0, mv0, p);
@@ -265,7 +285,8 @@ int augtree_plan_create(const augtree_desc_t *desc, int device, augtree_plan_t *
     r = cudaSetDevice(device) == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
     if (!r) r = pl->head_dim == 128 ? set_kernel_attributes<128>() : set_kernel_attributes<64>();
     try {
-      for (int k = 0; k < SCHED_COUNT && !r; ++k) r = upload_sched(pl->sched[k], pl->n_lanes);
+      for (int k = 0; k < SCHED_COUNT && !r; ++k)
+        r = upload_sched(pl->sched[k], pl->n_lanes, k == SCHED_REPLAY_FWD && (pl->flags & AUGTREE_FLAG_TEST_DROP_ITEM));
     } catch (...) {
       r = AUGTREE_ERR_INTERNAL;
     }
@@ -277,7 +298,8 @@ int augtree_plan_create(const augtree_desc_t *desc, int device, augtree_plan_t *
     if (!r) r = upload(pl->tiles_replay, &pl->d_tiles_replay);
     if (!r) r = upload(pl->tiles_prefill, &pl->d_tiles_prefill);
     if (!r) {
-      if (cudaMalloc(&pl->d_status, 2 * sizeof(int)) != cudaSuccess || cudaMemset(pl->d_status, 0, 2 * sizeof(int)) != cudaSuccess)
+      if (cudaMalloc(&pl->d_status, kStatusInts * sizeof(int)) != cudaSuccess ||
+          cudaMemset(pl->d_status, 0, kStatusInts * sizeof(int)) != cudaSuccess)
         r = AUGTREE_ERR_CUDA;
     }
     cudaSetDevice(prev);
@@ -490,6 +512,22 @@ int augtree_last_device_status(const augtree_plan_t *pl, int *status, int *detai
   if (e != cudaSuccess) return AUGTREE_ERR_CUDA;
   *status = h[0];
   if (detail) *detail = h[1];
+  return AUGTREE_OK;
+}
+
+int augtree_items_completed(const augtree_plan_t *pl, int kernel, long long *completed, long long *expected) {
+  int r = check_plan_any_device(pl);
+  if (r || kernel < 0 || kernel >= SCHED_COUNT || !completed || !expected) return AUGTREE_ERR_INVALID_ARG;
+  int prev = 0;
+  cudaGetDevice(&prev);
+  cudaSetDevice(pl->device);
+  int n = 0;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(&n, pl->d_status + 2 + kernel, sizeof(int), cudaMemcpyDeviceToHost);
+  cudaSetDevice(prev);
+  if (e != cudaSuccess) return AUGTREE_ERR_CUDA;
+  *completed = n;
+  *expected = pl->launched_items[kernel].load();
   return AUGTREE_OK;
 }
 

@@ -40,6 +40,9 @@ struct BwdParams {
   int causal_fp32;
   float scale, scale_log2;
   int *status;
+  long long wait_budget;    // clocks a wait may take before the kernel gives up
+  int kind;                 // schedule index: status[2 + kind] counts finished items
+  int test_flags;           // TEST_SKIP_BWD_LOAD: lane 0 never loads the first dO tile of its first item
 };
 
 constexpr int kBwdThreads = 576;  // 16 element-wise warps, TMA warp, MMA warp
@@ -110,7 +113,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tR0 = tmem, tR1 = tmem + 128, tDV = tmem + 256, tDK = tmem + 256 + D;
-  const AbortCtx ab{abort_flag, p.status};
+  const AbortCtx ab{abort_flag, p.status, p.wait_budget};
   const int rep = p.h_q / p.h_kv;
   const int it_begin = p.lane_ptr[blockIdx.x], it_end = p.lane_ptr[blockIdx.x + 1];
 
@@ -146,6 +149,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               for (int b = 0; b < NBOX; ++b) tma_load_3d(sQ0 + st * TILE + b * 16384, &tm_q, bar_q_full + 8 * st, b * 64, head, row);
               bulk_load_1d(sStats0 + st * 1024, p.stats + ((long long)head * p.n_tiles + s_tile0 + qt) * 256, 1024,
                            bar_q_full + 8 * st);
+              if ((p.test_flags & TEST_SKIP_BWD_LOAD) && blockIdx.x == 0 && T == 0) continue;  // injected fault
               ok = mbar_wait(bar_do_empty + 8 * st, par, ab, WAIT_BWD_QDO_EMPTY);
               if (!ok) break;
               mbar_expect_tx(bar_do_full + 8 * st, TILE);
@@ -400,6 +404,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       }
       tc_fence_before();
       warp_arrive(bar_acc_empty);
+      if (warp == 0 && lane == 0) atomicAdd(p.status + 2 + p.kind, 1);  // item finished (work accounting)
     }
   }
 

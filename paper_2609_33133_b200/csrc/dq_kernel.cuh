@@ -33,6 +33,8 @@ struct DqParams {
   int h_q;
   float scale, scale_log2;
   int *status;
+  long long wait_budget;    // clocks a wait may take before the kernel gives up
+  int kind;                 // schedule index: status[2 + kind] counts finished items
 };
 
 constexpr int kDqThreads = 320;
@@ -98,7 +100,7 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tQ = tmem, tDO = tmem + D / 2, tS = tmem + 128, tDP = tmem + 256, tDQ = tmem + 384;
-  const AbortCtx ab{abort_flag, p.status};
+  const AbortCtx ab{abort_flag, p.status, p.wait_budget};
   const int it_begin = p.lane_ptr[blockIdx.x], it_end = p.lane_ptr[blockIdx.x + 1];
 
   if (warp == 8) {
@@ -334,6 +336,7 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       }
       tc_fence_before();
       warp_arrive(bar_dq_empty);
+      if (warp == 0 && lane == 0) atomicAdd(p.status + 2 + p.kind, 1);  // item finished (work accounting)
     }
   }
 

@@ -34,6 +34,9 @@ struct FwdParams {
   float scale_log2;         // softmax scale * log2(e)
   const float *kmax2;       // [h_kv] largest squared key norm of the call's K tensors (key_norm_kernel)
   int *status;
+  long long wait_budget;    // clocks a wait may take before the kernel gives up
+  int kind;                 // schedule index: status[2 + kind] counts finished items
+  int test_flags;           // TEST_SKIP_FWD_LOAD: lane 0 never loads the first V tile of its first item
 };
 
 constexpr int kFwdThreads = 320;
@@ -110,7 +113,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const AbortCtx ab{abort_flag, p.status};
+  const AbortCtx ab{abort_flag, p.status, p.wait_budget};
   const int it_begin = p.lane_ptr[blockIdx.x], it_end = p.lane_ptr[blockIdx.x + 1];
 
   if (warp == 8) {
@@ -131,6 +134,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           for (int b = 0; b < NBOX; ++b) tma_load_3d(sQ + g * TILE + b * 16384, &tm_q, bar_q_full, b * 64, head, q_tok0 + g * 128);
         auto load_tile = [&](bool is_v, int j) -> bool {
           const uint32_t slot = kvc % NS, par = ((kvc / NS) & 1) ^ 1;
+          if ((p.test_flags & TEST_SKIP_FWD_LOAD) && blockIdx.x == 0 && ic == 0 && is_v && j == 0) { ++kvc; return true; }  // injected fault
           if (!mbar_wait(bar_kv_empty + 8 * slot, par, ab, WAIT_FWD_KV_EMPTY)) return false;
           const bool in_a = j < nA;
           const CUtensorMap *tm = in_a ? (is_v ? &tm_va : &tm_ka) : (is_v ? &tm_vb : &tm_kb);
@@ -506,6 +510,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         tc_fence_before();
         warp_arrive(bar_o_empty + 8 * g);
       }
+      if (ok && warp == 0 && lane == 0) atomicAdd(p.status + 2 + p.kind, 1);  // item finished (work accounting)
     }
 #if AUGTREE_TRACE
     if (warp == 1 && lane == 0)

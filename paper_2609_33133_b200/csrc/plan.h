@@ -1,5 +1,6 @@
 // Internal plan object: packing metadata on the host and its device copies.
 #pragma once
+#include <atomic>
 #include <cstdint>
 #include <vector>
 
@@ -13,6 +14,8 @@ constexpr int kTileKV = 128;  // keys per tile
 
 enum { SCHED_PREFILL_FWD = 0, SCHED_REPLAY_FWD = 1, SCHED_REPLAY_BWD = 2, SCHED_PREFILL_BWD = 3, SCHED_REPLAY_DQ = 4, SCHED_PREFILL_DQ = 5,
        SCHED_COUNT = 6 };
+
+constexpr int kStatusInts = 2 + SCHED_COUNT;
 
 struct Sched {
   int item_ints = 0;
@@ -49,7 +52,8 @@ struct augtree_plan {
   int32_t *d_seg_replay = nullptr, *d_seg_prefill = nullptr, *d_branch_group = nullptr, *d_group_splits = nullptr;
   int32_t *d_cu_r = nullptr;
   int32_t *d_tiles_replay = nullptr, *d_tiles_prefill = nullptr;
-  int *d_status = nullptr;  // [2]: status, detail
+  int *d_status = nullptr;  // [kStatusInts]: status, detail, then the items each schedule's kernel has finished
+  mutable std::atomic<long long> launched_items[augtree::SCHED_COUNT] = {};  // items handed to launches so far
   augtree::Timing *timing = nullptr;  // optional CUDA-event timing of the tile kernels
   size_t ws_fwd = 0, ws_bwd = 0;
 };

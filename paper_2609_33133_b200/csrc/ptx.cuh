@@ -63,9 +63,13 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 // that the other warp roles leave their loops too.
 struct AbortCtx {
   volatile int *flag;  // shared memory
-  int *status;         // global: [0] status, [1] detail
+  int *status;         // global: [0] status, [1] detail, [2 + k] items finished by the kernel of schedule k
+  long long budget;    // clocks one wait may take
 };
-constexpr long long kWaitBudgetClocks = 1ll << 31;
+constexpr long long kWaitBudgetClocks = 1ll << 31;      // about a second
+constexpr long long kWaitBudgetClocksTest = 1ll << 21;  // about a millisecond (AUGTREE_FLAG_TEST_SHORT_WAIT)
+// test hooks carried in the kernels' parameters (set from the plan's AUGTREE_FLAG_TEST_* flags)
+enum : int { TEST_SKIP_FWD_LOAD = 1, TEST_SKIP_BWD_LOAD = 2 };
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const AbortCtx &ab, int site) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -75,7 +79,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0) {
       if (*ab.flag) return false;
-      if (clock64() - t0 > kWaitBudgetClocks) {
+      if (clock64() - t0 > ab.budget) {
         *ab.flag = 1;
         if (atomicCAS(ab.status, 0, -5) == 0) ab.status[1] = site;
         return false;
