@@ -66,10 +66,41 @@ def peaks():
     return {"bf16_tflops": FALLBACK_BF16_TFLOPS, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture of this workload (the summary under
-# profiles/ gives the command); None for workloads that were not captured
-NCU_DRAM_BYTES = {("cfg2-7b-layer", "replay_bwd_dkdv"): 1.215e9, ("cfg2-7b-layer", "replay_bwd_dq"): 0.384e9,
-                  ("cfg2-7b-layer", "replay_fwd"): 0.254e9}
+def ncu_dram_bytes(workload, kernel):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch from the latest ncu capture of this workload
+    (profiles/ncu_dram_bytes.json, written from the capture whose command it records); None if not captured."""
+    path = os.path.join(ROOT, "profiles", "ncu_dram_bytes.json")
+    try:
+        return json.load(open(path)).get(workload, {}).get(kernel)
+    except (OSError, ValueError):
+        return None
+
+
+def algorithmic_bytes(w, kernel):
+    """HBM bytes a launch has to move if every tensor it touches crosses once (bf16 unless noted)."""
+    d, hq, hkv = w.head_dim, w.h_q, w.h_kv
+    tp, tr = w.total_prompt, w.total_response
+    q = lambda n: 2 * n * hq * d            # a query-sized bf16 tensor
+    kv = lambda n: 2 * n * hkv * d          # a key/value-sized bf16 tensor
+    stats = lambda n: 8 * n * hq            # fp32 lse*log2e and delta per (row, head)
+    return {
+        "prefill_fwd": q(tp) + 2 * kv(tp) + q(tp) + 4 * tp * hq,
+        "replay_fwd": q(tr) + 2 * kv(tr) + 2 * kv(tp) + q(tr) + 4 * tr * hq,
+        # Q, dO, statistics, K/V of both tensors in; dK_R, dV_R out; fp32 prompt accumulators read and written
+        "replay_bwd_dkdv": 2 * q(tr) + stats(tr) + 2 * kv(tr) + 2 * kv(tp) + 2 * kv(tr) + 2 * 2 * (2 * kv(tp)),
+        "prefill_bwd_dkdv": 2 * q(tp) + stats(tp) + 2 * kv(tp) + 2 * 2 * (2 * kv(tp)),
+        "replay_bwd_dq": 2 * q(tr) + stats(tr) + 2 * kv(tr) + 2 * kv(tp) + q(tr),
+        "prefill_bwd_dq": 2 * q(tp) + stats(tp) + 2 * kv(tp) + q(tp),
+    }[kernel]
+
+
+def config_record(w, world):
+    """The `config` object of the JSON line (the same keys for both arms)."""
+    fl = useful_flops(w)
+    return {"workload": w.name, "groups": w.n_groups, "prompt_tokens": w.total_prompt, "response_tokens": w.total_response,
+            "h_q": w.h_q, "h_kv": w.h_kv, "head_dim": w.head_dim, "useful_tflop_per_step": fl["total"] / 1e12,
+            "l2": "no flush: inputs + outputs exceed the 126 MB L2 (K/V reuse from L2 is part of the method)",
+            "parallelism": f"independent groups x{world}"}
 
 
 class ClockSampler:
@@ -161,7 +192,7 @@ def run_reference(args, w):
     val = fl["total"] / est / 1e12
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f64", "data": "synthetic", "config": {"workload": w.name, "tokens": w.total_prompt + w.total_response},
+            "dtype": "f64", "data": "synthetic", "config": config_record(w, 1),
             "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": info["cores"], "kind": "oracle",
                              "sample": f"{info['sequences']} of {info['of']} flattened (branch, head) sequences per step, time extrapolated"},
             "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -216,6 +247,83 @@ def time_steps(step_fn, steps, warmup, dist, sampler_index=None):
     return ms, (sampler.summary() if sampler else None)
 
 
+def measure_config(B, index, local_rank, steps=3, warmup=3, flattened=True):
+    """One of the other configurations, briefly: tree step, flattened step, clocks (rank 0, N = 1 only)."""
+    w = wl.config(index)
+    fl = useful_flops(w)
+    big = (w.total_prompt + w.total_response) * w.h_q * w.head_dim > 2e8
+    t = {k: v.cuda() for k, v in wl.make_tensors(w, device="cuda" if big else "cpu").items()}
+    splits = 4 if w.extra.get("force_split") else 0
+    plan = B.Plan(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, device=local_rank, flags=B.FLAG_ZERO_PROMPT_GRAD,
+                  kv_splits=splits)
+    out = B.alloc_outputs(plan)
+    ms, clocks = time_steps(lambda: B.run_forward_backward(plan, t, out), steps, warmup, None, sampler_index=local_rank)
+    ms /= steps
+    st = plan.device_status()
+    if st != (0, 0):
+        raise RuntimeError(f"device status {st} on configuration {index}")
+    rec = {"workload": w.name, "tokens": w.total_prompt + w.total_response, "useful_tflop_per_step": fl["total"] / 1e12,
+           "ms_per_step": ms, "tflops": fl["total"] / (ms * 1e-3) / 1e12, "steps": steps, "warmup": warmup,
+           "reuse_factor": fl["reuse_factor"], "sm_mhz": clocks["sm_mhz"], "reasons": clocks["reasons"], "kv_splits": splits}
+    del out
+    if flattened:
+        fw = w.flattened()
+        ft = wl.flatten_tensors(w, t)
+        del t
+        e = lambda h: torch.empty((0, h, w.head_dim), dtype=torch.bfloat16, device="cuda")
+        ft.update({"q_r": e(w.h_q), "k_r": e(w.h_kv), "v_r": e(w.h_kv), "do_r": e(w.h_q)})
+        fplan = B.Plan(fw.prompt_len, fw.branch_len, fw.h_q, fw.h_kv, fw.head_dim, device=local_rank, flags=B.FLAG_ZERO_PROMPT_GRAD)
+        fout = B.alloc_outputs(fplan)
+        fsteps = 2
+        fms, _ = time_steps(lambda: B.run_forward_backward(fplan, ft, fout), fsteps, 3, None)
+        fms /= fsteps
+        rec.update({"flattened_ms_per_step": fms, "speedup_vs_flattened": fms / ms, "meets_reuse_factor": bool(fms / ms >= fl["reuse_factor"])})
+        del fout, ft
+    torch.cuda.empty_cache()
+    return rec
+
+
+def run_strong(args, B, base, rank, world, local_rank, dist, pk):
+    """--scaling strong: ONE workload split over the ranks with no exchange step (whole groups, or (group, KV head)
+    pairs when there are fewer groups than ranks: workloads.partition).  Every rank generates the same seeded tensors
+    and keeps its parts' slices; `value` is the whole workload's useful FLOPs over the slowest rank's time."""
+    fl = useful_flops(base)
+    parts = wl.partition(base, world)[rank]
+    big = (base.total_prompt + base.total_response) * base.h_q * base.head_dim > 2e8
+    full = {k: v.cuda() for k, v in wl.make_tensors(base, device="cuda" if big else "cpu").items()}
+    jobs = []
+    for part in parts:
+        pw = wl.part_workload(base, part)
+        pt = wl.part_tensors(base, full, part)
+        plan = B.Plan(pw.prompt_len, pw.branch_len, pw.h_q, pw.h_kv, pw.head_dim, device=local_rank, flags=B.FLAG_ZERO_PROMPT_GRAD,
+                      kv_splits=4 if pw.extra.get("force_split") else 0)
+        jobs.append((pw, plan, pt, B.alloc_outputs(plan)))
+    del full
+
+    def step():
+        for _, plan, pt, out in jobs:
+            B.run_forward_backward(plan, pt, out)
+
+    l0 = B.launch_count()
+    ms, clocks = time_steps(step, args.steps, args.warmup, dist, sampler_index=local_rank if rank == 0 else None)
+    launches = (B.launch_count() - l0) // (args.steps + args.warmup) * args.steps
+    for _, plan, _, _ in jobs:
+        if plan.device_status() != (0, 0):
+            raise RuntimeError("device status")
+    ms_step = ms / args.steps
+    mine = sum(useful_flops(pw)["total"] for pw, _, _, _ in jobs)
+    if rank == 0:
+        value = fl["total"] / (ms_step * 1e-3) / 1e12
+        line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16",
+                "data": "synthetic", "config": {**config_record(base, 1), "parallelism": f"one workload over {world} ranks: "
+                                                "whole groups or (group, KV head) units, no exchange step"},
+                "rank0_share_of_flops": mine / fl["total"], "rank0_parts": [[p.groups, p.kv_heads] for p in parts],
+                "pct_of_measured_bf16_peak": 100 * value / world / pk["bf16_tflops"], "gpu_launches": int(launches), "clocks": clocks,
+                "e2e": None, "roofline": None, "cpu_baseline": None}
+        print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -226,6 +334,9 @@ def main():
     ap.add_argument("--no-flattened", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-configs", action="store_true", help="skip the brief runs of the other four configurations")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="weak (default): every rank runs its own groups; strong: one workload partitioned over the ranks")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -249,9 +360,15 @@ def main():
         import torch.distributed as dist_mod
         dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
         dist = dist_mod
+    pk = peaks()
+    if args.scaling == "strong":
+        run_strong(args, B, w, rank, world, local_rank, dist, pk)
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return 0
     w = rank_workload(w, rank)
     fl = useful_flops(w)
-    pk = peaks()
 
     big = (w.total_prompt + w.total_response) * w.h_q * w.head_dim > 2e8
     t_dev = wl.make_tensors(w, device="cuda" if big else "cpu")
@@ -295,7 +412,8 @@ def main():
     dom = max(per_kernel, key=lambda n: per_kernel[n]["ms"])
     roofline = {"bound": "tensor", "kernel": f"{kfun[dom]} ({dom})", "achieved": per_kernel[dom]["tflops"],
                 "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": per_kernel[dom]["tflops"] / pk["bf16_tflops"],
-                "peak_source": f"{pk['source']} cuBLAS bf16 burst", "traffic": NCU_DRAM_BYTES.get((w.name, dom)),
+                "peak_source": f"{pk['source']} cuBLAS bf16 burst", "traffic": ncu_dram_bytes(w.name, dom),
+                "algorithmic_bytes": algorithmic_bytes(w, dom),
                 # the kernel is timed inside a loop of steps that runs under the power cap; against the sustained figure:
                 "peak_sustained": pk["bf16_tflops_sustained"], "frac_sustained": per_kernel[dom]["tflops"] / pk["bf16_tflops_sustained"]}
 
@@ -343,21 +461,31 @@ def main():
         cpu = {"value": fl["total"] / info["est_total_s"] / 1e12, "unit": "TFLOP/s", "cores": info["cores"], "kind": "oracle",
                "sample": f"{info['sequences']} of {info['of']} flattened (branch, head) sequences, {info['seconds_sample']:.1f} s, extrapolated"}
 
+    # ---- the other four configurations, briefly (3 timed steps each; `value` stays the default workload's)
+    others = None
+    if rank == 0 and world == 1 and args.config == 2 and not args.no_configs:
+        del out, t_dev
+        torch.cuda.empty_cache()
+        others = {}
+        for index in (1, 3, 4, 5):
+            try:
+                others[f"cfg{index}"] = measure_config(B, index, local_rank)
+            except (RuntimeError, torch.OutOfMemoryError) as exc:   # reported, not fatal: the headline line still prints
+                others[f"cfg{index}"] = {"error": str(exc)[:200]}
+                torch.cuda.empty_cache()
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": per_step[0],
             "plan_create_ms": plan_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": {"workload": w.name, "groups": w.n_groups, "prompt_tokens": w.total_prompt, "response_tokens": w.total_response,
-                       "h_q": w.h_q, "h_kv": w.h_kv, "head_dim": w.head_dim, "useful_tflop_per_step": fl["total"] / 1e12,
-                       "l2": "no flush: inputs + outputs exceed the 126 MB L2 (K/V reuse from L2 is part of the method)",
-                       "parallelism": f"independent groups x{world}"},
+            "config": config_record(w, world),
             "pct_of_measured_bf16_peak": 100 * value / world / pk["bf16_tflops"],
             "pct_of_measured_bf16_sustained": 100 * value / world / pk["bf16_tflops_sustained"],
             "pct_of_nominal_bf16_peak": 100 * value / world / NOMINAL_BF16_TFLOPS,
             "kernels": per_kernel, "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
-            "flattened": flat, "cpu_baseline": cpu,
+            "flattened": flat, "cpu_baseline": cpu, "configs": others,
         }
         print(json.dumps(line), flush=True)
     if dist is not None:

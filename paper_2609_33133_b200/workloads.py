@@ -126,6 +126,103 @@ def config5_prefix_256k() -> Workload:
 TENSOR_NAMES = ("q_p", "k_p", "v_p", "do_p", "q_r", "k_r", "v_r", "do_r")
 
 
+# --------------------------------------------------------------------------- #
+# Sharding over GPUs without any exchange step.  Replay trees are independent of
+# each other (the paper's CP groups "run different trees", Sec. 3.5) and, inside
+# attention, so are KV heads: a KV head with the query heads that read it can live
+# on one GPU, and the many-to-one prompt-KV gradient of Eq. 2 stays local to it.
+# So the units are whole groups when there are at least as many groups as ranks,
+# and (group, KV head) pairs otherwise; they are dealt out largest first by visible
+# (query, key) pairs, each to the rank with the least work so far.
+@dataclass
+class Part:
+    """Some groups of a workload, restricted to some of its KV heads (and their query heads)."""
+    groups: List[int]
+    kv_heads: List[int]
+
+
+def _group_pairs(w: Workload, g: int) -> int:
+    tri = lambda n: n * (n + 1) // 2
+    p = w.prompt_len[g]
+    return tri(p) + sum(r * p + tri(r) for r in w.branch_len[g])
+
+
+def partition(w: Workload, world: int) -> List[List[Part]]:
+    """Parts per rank.  Every (group, KV head) of `w` lands in exactly one part of exactly one rank."""
+    all_heads = list(range(w.h_kv))
+    if w.n_groups >= world:
+        units = [(g, None) for g in range(w.n_groups)]
+        weight = lambda u: _group_pairs(w, u[0]) * w.h_kv
+    else:
+        units = [(g, c) for g in range(w.n_groups) for c in all_heads]
+        weight = lambda u: _group_pairs(w, u[0])
+    order = sorted(range(len(units)), key=lambda i: (-weight(units[i]), i))
+    load = [0] * world
+    mine: List[List[tuple]] = [[] for _ in range(world)]
+    for i in order:
+        r = min(range(world), key=lambda k: (load[k], k))
+        mine[r].append(units[i])
+        load[r] += weight(units[i])
+    shards = []
+    for r in range(world):
+        whole = sorted(g for g, c in mine[r] if c is None)
+        parts = [Part(whole, all_heads)] if whole else []
+        by_heads = {}
+        for g in sorted({g for g, c in mine[r] if c is not None}):
+            heads = tuple(sorted(c for gg, c in mine[r] if gg == g and c is not None))
+            by_heads.setdefault(heads, []).append(g)
+        parts += [Part(gs, list(heads)) for heads, gs in sorted(by_heads.items())]
+        shards.append(parts)
+    return shards
+
+
+def part_workload(w: Workload, part: Part) -> Workload:
+    rep = w.h_q // w.h_kv
+    return Workload(f"{w.name}[g{part.groups},kv{part.kv_heads}]", [w.prompt_len[g] for g in part.groups],
+                    [list(w.branch_len[g]) for g in part.groups], rep * len(part.kv_heads), len(part.kv_heads), w.head_dim,
+                    w.seed, w.note, dict(w.extra))
+
+
+def _part_index(w: Workload, part: Part):
+    """(prompt token index, response token index, query head index, KV head index) of a part inside `w`."""
+    cu_p = np.concatenate([[0], np.cumsum(w.prompt_len)])
+    flat = [sum(b) for b in w.branch_len]
+    cu_r = np.concatenate([[0], np.cumsum(flat)])
+    tok_p = np.concatenate([np.arange(cu_p[g], cu_p[g + 1]) for g in part.groups]) if part.groups else np.zeros(0, int)
+    tok_r = np.concatenate([np.arange(cu_r[g], cu_r[g + 1]) for g in part.groups]) if part.groups else np.zeros(0, int)
+    rep = w.h_q // w.h_kv
+    hq = np.concatenate([np.arange(c * rep, (c + 1) * rep) for c in part.kv_heads])
+    return tok_p.astype(np.int64), tok_r.astype(np.int64), hq.astype(np.int64), np.asarray(part.kv_heads, dtype=np.int64)
+
+
+def part_tensors(w: Workload, t, part: Part):
+    """The part's slices of a workload's tensors (copies; pure data movement)."""
+    tok_p, tok_r, hq, hkv = _part_index(w, part)
+    out = {}
+    for name in TENSOR_NAMES:
+        x = t[name]
+        tok = torch.as_tensor(tok_p if name.endswith("_p") else tok_r, device=x.device)
+        heads = torch.as_tensor(hq if name[0] in "qd" else hkv, device=x.device)
+        out[name] = x.index_select(0, tok).index_select(1, heads).contiguous()
+    return out
+
+
+def scatter_part(w: Workload, part: Part, part_out, full_out):
+    """Writes a part's outputs (any of o_*, lse_*, dq_*, dk_*, dv_*) into full-size tensors of `w`."""
+    tok_p, tok_r, hq, hkv = _part_index(w, part)
+    for name, x in part_out.items():
+        if name not in full_out:
+            continue
+        dst = full_out[name]
+        tok = torch.as_tensor(tok_p if name.endswith("_p") else tok_r, device=dst.device)
+        q_like = name.startswith(("o_", "lse_", "dq_"))
+        heads = torch.as_tensor(hq if q_like else hkv, device=dst.device)
+        if name.startswith("lse"):
+            dst[heads[:, None], tok[None, :]] = x.to(dst.device)
+        else:
+            dst[tok[:, None], heads[None, :]] = x.to(dst.device)
+
+
 def make_tensors(w: Workload, device="cpu"):
     """bf16 tensors ~ N(0,1) for a workload, from torch's seeded generator.
 

@@ -113,6 +113,23 @@ def test_results_are_bitwise_repeatable(B):
         assert np.array_equal(a[k], b[k]), k
 
 
+def test_kv_head_shards_reproduce_the_unsharded_result_bitwise(B):
+    """Strong-scaling shards need no exchange: configuration 1 split into two KV-head shards (workloads.partition),
+    run one after the other, gives bit for bit the outputs of the unsharded run, prompt-KV gradients included."""
+    w = wl.config(1)
+    t = wl.make_tensors(w)
+    whole, _ = pu.run_gpu(B, w, t)
+    shards = wl.partition(w, 2)
+    assert [len(s) for s in shards] == [1, 1] and sorted(shards[0][0].kv_heads + shards[1][0].kv_heads) == [0, 1, 2, 3]
+    joined = {k: torch.full(v.shape, float("nan"), dtype=torch.float64) for k, v in ((k, torch.from_numpy(v)) for k, v in whole.items())}
+    for parts in shards:
+        for part in parts:
+            got, _ = pu.run_gpu(B, wl.part_workload(w, part), wl.part_tensors(w, t, part))
+            wl.scatter_part(w, part, {k: torch.from_numpy(v) for k, v in got.items()}, joined)
+    for k in whole:
+        assert np.array_equal(joined[k].numpy(), whole[k]), k
+
+
 def test_flattened_baseline_matches_tree(B):
     """The no-reuse baseline (same kernels, prompt duplicated per branch) gives the tree's results;
     its per-copy prompt gradients add up to the tree's (Eq. 2)."""

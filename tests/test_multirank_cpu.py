@@ -51,6 +51,50 @@ def test_two_gloo_ranks_shard_and_reduce():
     assert all(abs(r[4] - 2 * fl / 15e-3 / 1e12) < 1e-9 for r in res)  # whole-job value over the slowest rank's time
 
 
+def _partition_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    res = {}
+    for index in (1, 2, 3, 5):
+        w = wl.config(index)
+        mine = wl.partition(w, world)[rank]
+        units = [(g, c) for part in mine for g in part.groups for c in part.kv_heads]
+        flops = sum(bench.useful_flops(wl.part_workload(w, part))["total"] for part in mine)
+        gathered = [None] * world
+        dist.all_gather_object(gathered, (units, flops))          # the only cross-rank step: bookkeeping, not data
+        res[index] = gathered
+    out.put((rank, res))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_partition_covers_every_group_and_kv_head_once_on_two_ranks():
+    """Strong-scaling shards (whole groups, or (group, KV head) units when groups < ranks): every unit on exactly one
+    rank, the ranks' useful FLOPs add up to the workload's, and both ranks see the same answer."""
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_partition_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = dict(q.get(timeout=180) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res[0] == res[1]
+    for index, gathered in res[0].items():
+        w = wl.config(index)
+        units = [u for us, _ in gathered for u in us]
+        assert sorted(units) == [(g, c) for g in range(w.n_groups) for c in range(w.h_kv)], index
+        assert sum(f for _, f in gathered) == bench.useful_flops(w)["total"], index
+        loads = [f for _, f in gathered]
+        assert max(loads) <= 0.56 * sum(loads), (index, loads)     # largest-first keeps two ranks within a few percent
+    # fewer units than ranks: the extra ranks get nothing, nothing is lost
+    w = wl.config(2)
+    shards = wl.partition(w, 8)
+    assert sum(len(s) for s in shards) == 4 and sum(1 for s in shards if not s) == 4
+
+
 def test_flop_accounting_matches_oracle_pair_count():
     from oracle import tree_attention as ora
     for i in (1, 2, 3):
