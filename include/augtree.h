@@ -316,6 +316,62 @@ int augtree_assign_grid(const int64_t *weight, const int64_t *size, int n_units,
                         int64_t cell_cap, int exact_max_units, int32_t *round_out, int32_t *lane_out,
                         int64_t *critical_path, int32_t *solved_exactly);
 
+/*
+ * Online strategy planner (Sec. 3.4 "Online Strategy Planner", Algorithm 1, Eq. 6-10).  Host only, no device work.
+ * For one replay tree T = (P, {R_i}) and a set of candidate CP degrees it enumerates the candidates
+ * c = (d, pi, (b, s), X): per degree d the fused candidate (RingCP, b = 0: ordinary ring CP over every (P, R_i) pair,
+ * the prompt recomputed per branch) and, for pi in {TreeMoveKV, MoveQ}, every lane count s that divides d (s <= G) and
+ * every round count b = 1 .. min(b_max, ceil(G / s)).  The replay units are the G response paths, unit k with weight
+ * w_k = its valid Q-KV tile count in replay (128 x 128 tiles: query tiles x prompt tiles + its causal triangle) and size
+ * R_k tokens; X comes from the AssignGrid step (augtree_assign_grid: exact up to exact_max_units units, largest-first
+ * above) under the cell limit the memory model gives.  Each feasible candidate is scored with Eq. 7,
+ *   T(c) = gamma_c (T_prefill + T_replay),
+ *   Eq. 8   T_prefill = alpha_p L_P / d_eff + beta_p L_P f_ring(d_eff) + lat_p0 + lat_p1 d_eff
+ *           (d_eff = d for MoveQ; d_lane = d / s for TreeMoveKV, where every lane prefills the prompt itself),
+ *   Eq. 9   TreeMoveKV: alpha_tmkv W / d_lane + beta_tmkv C_KV + lat_tmkv0 + lat_tmkv1 b d_lane,
+ *           C_KV = b 2 (L_P + L_cell) H_kv f_ring(d_lane)                                        (Eq. 3 per round),
+ *   Eq. 10  MoveQ: alpha_mq W / d_lane + beta_q C_Q + T_r + lat_mq0 + lat_mq1 b,
+ *           C_Q = b L_cell H_q (Eq. 4),  T_r = b (red0 + red1 L_cell H_q) f_ring(d),
+ *   b = 0   gamma_ring sum_i [alpha_ring tiles(L_P + R_i) / d + beta_ring 2 (L_P + R_i) H_kv f_ring(d) + lat_ring0 + lat_ring1 d],
+ * with W the critical-path work of X (Eq. 6's objective), f_ring(d) = (d - 1) / d, and L_cell = ceil(G / (b s)) max_i R_i,
+ * the paper's conservative replay-length proxy applied to a cell.  Per-rank memory (mem_cap <= 0: no limit):
+ * TreeMoveKV  mem_prompt L_P / d_lane + mem_resp cell_tokens / d_lane <= mem_cap;  MoveQ  mem_prompt L_P / d +
+ * mem_resp cell_tokens / d_lane <= mem_cap;  RingCP  (mem_prompt L_P + mem_resp max_i R_i) / d <= mem_cap.
+ * The paper gives the form of these terms and leaves every constant to profiling, so all constants are inputs; the
+ * definitions of f_ring, L_cell, T_r and the memory shares are this library's readings of what the paper leaves open.
+ * Ties go to the candidate enumerated first (degrees in the given order, RingCP, TreeMoveKV, MoveQ, s ascending, b
+ * ascending).  round_out / lane_out [n_branches] receive X of the chosen candidate (zeros for RingCP).  Returns
+ * AUGTREE_ERR_UNSUPPORTED when no candidate is feasible.  All pointers are host memory owned by the caller.
+ */
+enum { AUGTREE_RING_CP = 0, AUGTREE_TREE_MOVE_KV = 1, AUGTREE_MOVE_Q = 2 };
+typedef struct {
+  double alpha_p, beta_p, lat_p0, lat_p1;
+  double alpha_tmkv, beta_tmkv, lat_tmkv0, lat_tmkv1;
+  double alpha_mq, beta_q, red0, red1, lat_mq0, lat_mq1;
+  double alpha_ring, beta_ring, lat_ring0, lat_ring1;
+  double gamma_ring, gamma_tmkv, gamma_mq;
+  double mem_cap, mem_prompt, mem_resp;
+} augtree_profile_t;
+typedef struct {
+  uint32_t struct_size;        /* sizeof(augtree_tree_t)                                  */
+  int32_t prompt_len;          /* L_P >= 1                                                */
+  int32_t n_branches;          /* G >= 0                                                  */
+  const int32_t *branch_len;   /* [G] R_i >= 1                                     (host) */
+  int32_t h_q, h_kv;
+  int32_t n_degrees;
+  const int32_t *degrees;      /* [n_degrees] candidate CP degrees d >= 1          (host) */
+  int32_t b_max;               /* most rounds tried; 0 selects 4                          */
+  int32_t exact_max_units;     /* as in augtree_assign_grid; 0 selects 12                 */
+} augtree_tree_t;
+typedef struct {
+  double cost;                 /* T(c*) by Eq. 7                                          */
+  int32_t degree, primitive, rounds, lanes;   /* d, pi, b, s of c*                        */
+  int32_t solved_exactly;      /* 1: X of c* is an exact minimum of Eq. 6                 */
+  int32_t n_candidates;        /* candidates enumerated                                   */
+} augtree_choice_t;
+int augtree_plan_tree(const augtree_tree_t *tree, const augtree_profile_t *profile, augtree_choice_t *choice,
+                      int32_t *round_out, int32_t *lane_out);
+
 const char *augtree_status_string(int status);
 
 #ifdef __cplusplus

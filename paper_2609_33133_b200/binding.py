@@ -33,7 +33,7 @@ EXPORTS = ["augtree_plan_create", "augtree_plan_destroy", "augtree_plan_workspac
            "augtree_prefill_fwd", "augtree_replay_fwd", "augtree_replay_bwd", "augtree_prefill_bwd",
            "augtree_last_device_status", "augtree_launch_count", "augtree_status_string",
            "augtree_set_timing", "augtree_get_kernel_time", "augtree_replay_fwd_static", "augtree_assign_grid",
-           "augtree_items_completed"]
+           "augtree_items_completed", "augtree_plan_tree"]
 
 
 class Desc(C.Structure):
@@ -45,6 +45,7 @@ class Desc(C.Structure):
 
 
 _vp, _sz = C.c_void_p, C.c_size_t
+_i64p, _i32p = C.POINTER(C.c_int64), C.POINTER(C.c_int32)
 lib.augtree_plan_create.argtypes = [C.POINTER(Desc), C.c_int, C.POINTER(_vp)]
 lib.augtree_plan_destroy.argtypes = [_vp]
 lib.augtree_plan_workspace_bytes.argtypes = [_vp, C.POINTER(_sz), C.POINTER(_sz)]
@@ -63,8 +64,46 @@ lib.augtree_status_string.restype = C.c_char_p
 lib.augtree_status_string.argtypes = [C.c_int]
 
 
-_i64p, _i32p = C.POINTER(C.c_int64), C.POINTER(C.c_int32)
 lib.augtree_assign_grid.argtypes = [_i64p, _i64p, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int, _i32p, _i32p, _i64p, _i32p]
+
+
+PROFILE_FIELDS = ["alpha_p", "beta_p", "lat_p0", "lat_p1", "alpha_tmkv", "beta_tmkv", "lat_tmkv0", "lat_tmkv1", "alpha_mq", "beta_q",
+                  "red0", "red1", "lat_mq0", "lat_mq1", "alpha_ring", "beta_ring", "lat_ring0", "lat_ring1", "gamma_ring",
+                  "gamma_tmkv", "gamma_mq", "mem_cap", "mem_prompt", "mem_resp"]
+RING_CP, TREE_MOVE_KV, MOVE_Q = 0, 1, 2
+
+
+class ProfileC(C.Structure):
+    _fields_ = [(n, C.c_double) for n in PROFILE_FIELDS]
+
+
+class TreeC(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("prompt_len", C.c_int32), ("n_branches", C.c_int32), ("branch_len", _i32p),
+                ("h_q", C.c_int32), ("h_kv", C.c_int32), ("n_degrees", C.c_int32), ("degrees", _i32p), ("b_max", C.c_int32),
+                ("exact_max_units", C.c_int32)]
+
+
+class ChoiceC(C.Structure):
+    _fields_ = [("cost", C.c_double), ("degree", C.c_int32), ("primitive", C.c_int32), ("rounds", C.c_int32),
+                ("lanes", C.c_int32), ("solved_exactly", C.c_int32), ("n_candidates", C.c_int32)]
+
+
+lib.augtree_plan_tree.argtypes = [C.POINTER(TreeC), C.POINTER(ProfileC), C.POINTER(ChoiceC), _i32p, _i32p]
+
+
+def plan_tree(prompt_len, branch_len, h_q, h_kv, degrees, profile: dict, b_max=0, exact_max_units=0):
+    """augtree_plan_tree: returns a dict with cost, degree, primitive, rounds, lanes, solved_exactly, n_candidates and the
+    placement X as (round[k], lane[k]).  `profile` maps the names in PROFILE_FIELDS to floats (missing: 0)."""
+    G = len(branch_len)
+    bl = (C.c_int32 * max(G, 1))(*[int(x) for x in branch_len])
+    dg = (C.c_int32 * len(degrees))(*[int(x) for x in degrees])
+    tree = TreeC(C.sizeof(TreeC), int(prompt_len), G, bl, h_q, h_kv, len(degrees), dg, b_max, exact_max_units)
+    prof = ProfileC(*[float(profile.get(n, 0.0)) for n in PROFILE_FIELDS])
+    ch = ChoiceC()
+    rounds, lanes = (C.c_int32 * max(G, 1))(), (C.c_int32 * max(G, 1))()
+    _check(lib.augtree_plan_tree(C.byref(tree), C.byref(prof), C.byref(ch), rounds, lanes), "augtree_plan_tree")
+    return {"cost": ch.cost, "degree": ch.degree, "primitive": ch.primitive, "rounds": ch.rounds, "lanes": ch.lanes,
+            "solved_exactly": bool(ch.solved_exactly), "n_candidates": ch.n_candidates, "X": (list(rounds[:G]), list(lanes[:G]))}
 
 
 class AugtreeError(RuntimeError):

@@ -6,6 +6,7 @@
 // size.  Up to `exact_max_units` units the minimum is found exactly by dynamic programming
 // over subsets (the paper's bounded AssignGrid); above it units are placed largest first.
 #include <algorithm>
+#include <cmath>
 #include <cstdint>
 #include <limits>
 #include <numeric>
@@ -165,6 +166,137 @@ extern "C" int augtree_assign_grid(const int64_t *weight, const int64_t *size, i
   try {
     return assign_grid_impl(weight, size, n_units, n_rounds, n_lanes, cell_cap, exact_max_units, round_out, lane_out,
                             critical_path, solved_exactly);
+  } catch (...) {
+    return AUGTREE_ERR_INTERNAL;
+  }
+}
+
+// --------------------------------------------------------------------------------------------------------------
+// Online strategy planner (Sec. 3.4, Algorithm 1): for one replay tree, enumerate the candidates c = (d, pi, (b, s), X)
+// over the given CP degrees, place the replay units (one per response path, weight = valid Q-KV tile count) with
+// AssignGrid, score each candidate with Eq. 7-10 and return the cheapest feasible one.  The paper leaves the constants
+// of the cost model to profiling: they are inputs.  Readings of what it leaves open (all stated in the header):
+// f_ring(d) = (d - 1) / d; lane counts s | d with s <= G; rounds b <= min(b_max, ceil(G / s)); the traffic terms use the
+// conservative proxy ceil(G / (b s)) * max_i R_i for the tokens of a cell, so that the placement enters through the
+// critical-path work W alone; per-rank memory = prompt share + cell share.
+namespace {
+
+constexpr int kTile = 128;
+inline int64_t cdiv64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline double f_ring(int d) { return (double)(d - 1) / (double)d; }
+inline int64_t replay_tiles(int64_t P, int64_t R) {
+  const int64_t nq = cdiv64(R, kTile);
+  return nq * cdiv64(P, kTile) + nq * (nq + 1) / 2;
+}
+inline int64_t causal_tiles(int64_t n) {
+  const int64_t nq = cdiv64(n, kTile);
+  return nq * (nq + 1) / 2;
+}
+
+}  // namespace
+
+static int plan_tree_impl(const augtree_tree_t *t, const augtree_profile_t *pr, augtree_choice_t *choice, int32_t *round_out,
+                          int32_t *lane_out) {
+  if (!t || !pr || !choice || t->struct_size != sizeof(augtree_tree_t)) return AUGTREE_ERR_INVALID_ARG;
+  const int G = t->n_branches;
+  if (t->prompt_len < 1 || G < 0 || (G > 0 && (!t->branch_len || !round_out || !lane_out))) return AUGTREE_ERR_INVALID_ARG;
+  if (t->n_degrees < 1 || !t->degrees || t->h_q < 1 || t->h_kv < 1) return AUGTREE_ERR_INVALID_ARG;
+  const int b_max = t->b_max > 0 ? t->b_max : 4;
+  const int64_t P = t->prompt_len;
+  std::vector<int64_t> w(G), m(G);
+  int64_t r_max = 0;
+  for (int k = 0; k < G; ++k) {
+    if (t->branch_len[k] < 1) return AUGTREE_ERR_INVALID_ARG;
+    m[k] = t->branch_len[k];
+    w[k] = replay_tiles(P, m[k]);
+    r_max = std::max(r_max, m[k]);
+  }
+  bool have = false;
+  augtree_choice_t best = {};
+  std::vector<int32_t> rounds(G), lanes(G), best_rounds(G), best_lanes(G);
+  int n_cand = 0;
+  for (int di = 0; di < t->n_degrees; ++di) {
+    const int d = t->degrees[di];
+    if (d < 1 || d > 65536) return AUGTREE_ERR_INVALID_ARG;
+    // ---- b = 0: ordinary ring CP over every (P, R_i) pair
+    {
+      ++n_cand;
+      const int64_t longest = P + r_max;
+      const bool fits = pr->mem_cap <= 0 || (pr->mem_prompt * (double)P + pr->mem_resp * (double)(longest - P)) / d <= pr->mem_cap;
+      if (fits) {
+        double total = 0.0;
+        for (int k = 0; k < std::max(G, 1); ++k) {
+          const int64_t r = G ? m[k] : 0;
+          total += pr->alpha_ring * (double)causal_tiles(P + r) / d + pr->beta_ring * 2 * (double)(P + r) * t->h_kv * f_ring(d) +
+                   pr->lat_ring0 + pr->lat_ring1 * d;
+        }
+        const double cost = pr->gamma_ring * total;
+        if (!have || cost < best.cost) {
+          have = true;
+          best.cost = cost; best.degree = d; best.primitive = AUGTREE_RING_CP; best.rounds = 0; best.lanes = 1; best.solved_exactly = 1;
+        }
+      }
+    }
+    if (G == 0) continue;
+    for (int primitive = AUGTREE_TREE_MOVE_KV; primitive <= AUGTREE_MOVE_Q; ++primitive)
+      for (int s = 1; s <= d && s <= G; ++s) {
+        if (d % s) continue;
+        const int d_lane = d / s;
+        // cell limit in response tokens from the per-rank memory model
+        int64_t cap = 0;  // 0: none
+        if (pr->mem_cap > 0) {
+          const double room = primitive == AUGTREE_TREE_MOVE_KV ? pr->mem_cap * d_lane - pr->mem_prompt * (double)P
+                                                                : (pr->mem_cap - pr->mem_prompt * (double)P / d) * d_lane;
+          if (room < 0) { n_cand += (int)std::min<int64_t>(b_max, cdiv64(G, s)); continue; }
+          cap = (int64_t)std::floor(room / pr->mem_resp);
+          if (cap < 1) { n_cand += (int)std::min<int64_t>(b_max, cdiv64(G, s)); continue; }   // not even one token fits
+        }
+        for (int b = 1; b <= std::min<int64_t>(b_max, cdiv64(G, s)); ++b) {
+          ++n_cand;
+          int64_t work = 0;
+          int32_t exact = 0;
+          const int r = assign_grid_impl(w.data(), m.data(), G, b, s, cap, t->exact_max_units, rounds.data(), lanes.data(), &work, &exact);
+          if (r == AUGTREE_ERR_UNSUPPORTED) continue;  // the units do not fit this grid
+          if (r) return r;
+          const double L = (double)(cdiv64(G, (int64_t)b * s) * r_max);
+          double replay, gamma;
+          int d_eff;
+          if (primitive == AUGTREE_TREE_MOVE_KV) {
+            d_eff = d_lane;
+            const double c_kv = b * 2 * ((double)P + L) * t->h_kv * f_ring(d_lane);
+            replay = pr->alpha_tmkv * (double)work / d_lane + pr->beta_tmkv * c_kv + pr->lat_tmkv0 + pr->lat_tmkv1 * b * d_lane;
+            gamma = pr->gamma_tmkv;
+          } else {
+            d_eff = d;
+            const double c_q = b * L * t->h_q;
+            const double t_r = b * (pr->red0 + pr->red1 * L * t->h_q) * f_ring(d);
+            replay = pr->alpha_mq * (double)work / d_lane + pr->beta_q * c_q + t_r + pr->lat_mq0 + pr->lat_mq1 * b;
+            gamma = pr->gamma_mq;
+          }
+          const double prefill = pr->alpha_p * (double)P / d_eff + pr->beta_p * (double)P * f_ring(d_eff) + pr->lat_p0 + pr->lat_p1 * d_eff;
+          const double cost = gamma * (prefill + replay);
+          if (!have || cost < best.cost) {
+            have = true;
+            best.cost = cost; best.degree = d; best.primitive = primitive; best.rounds = b; best.lanes = s; best.solved_exactly = exact;
+            best_rounds = rounds; best_lanes = lanes;
+          }
+        }
+      }
+  }
+  if (!have) return AUGTREE_ERR_UNSUPPORTED;
+  best.n_candidates = n_cand;
+  *choice = best;
+  for (int k = 0; k < G; ++k) {
+    round_out[k] = best.primitive == AUGTREE_RING_CP ? 0 : best_rounds[k];
+    lane_out[k] = best.primitive == AUGTREE_RING_CP ? 0 : best_lanes[k];
+  }
+  return AUGTREE_OK;
+}
+
+extern "C" int augtree_plan_tree(const augtree_tree_t *tree, const augtree_profile_t *profile, augtree_choice_t *choice,
+                                 int32_t *round_out, int32_t *lane_out) {
+  try {
+    return plan_tree_impl(tree, profile, choice, round_out, lane_out);
   } catch (...) {
     return AUGTREE_ERR_INTERNAL;
   }
