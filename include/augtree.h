@@ -268,6 +268,40 @@ int augtree_replay_fwd_static(const augtree_plan_t *plan, const void *q_r, const
 int augtree_last_device_status(const augtree_plan_t *plan, int *status, int *detail);
 
 /*
+ * Building blocks of context-parallel replay (Sec. 3.3 "Common tile semantics", MoveQ and TreeMoveKV).  A rank
+ * that holds one shard of the keys computes, for every response query it is given, the PARTIAL online-softmax
+ * state over that shard; the states of a query are merged afterwards (the (+) of Sec. 3.3), on whichever rank
+ * owns the query; in the backward pass every shard owner computes its shard's dK, dV and its contribution to dQ
+ * from the merged LSE, and the dQ contributions are summed on the way back ("its custom autograd operator applies
+ * the reverse communication", Sec. 3.3).  These three calls are the per-rank compute steps; moving queries,
+ * states and gradients between ranks is the caller's (NCCL or peer copies, no multicast loads).
+ *
+ * The plan describes THIS RANK'S view: its "prompt" is the shard of unmasked keys it holds (k_p, v_p: a prompt-KV
+ * shard, or any keys every given query may see in full), its branches are the response queries it is given.
+ * The plan must not use kv_splits.
+ *
+ * augtree_replay_fwd_state: state_o [sumR,H_q,d] fp32 (normalised partial output) and state_lse [H_q,sumR] fp32
+ *   over the keys {the plan's prompt} and, if include_own != 0, the query's own causal response prefix (k_r, v_r).
+ *   The state is kept as (normalised O, LSE): the same information as (m, l, O_acc).
+ * augtree_merge_states: merges n_states <= 16 such states (HOST arrays of DEVICE pointers) into o_r (bf16) and
+ *   lse_r; a state whose LSE is -inf (no key seen) has weight zero.
+ * augtree_replay_bwd_state: with the MERGED o_r, lse_r and the seed do_r: dkp_acc, dvp_acc += gradients of the
+ *   plan's prompt keys over all given queries (complete for this shard: Eq. 2's sum is local to the shard's owner);
+ *   dq_part [sumR,H_q,d] fp32 = this shard's contribution to dQ (written, not added); with include_own != 0 also
+ *   the own-response part: dk_r, dv_r (bf16) written and the causal range included in dq_part; with
+ *   include_own == 0, dk_r and dv_r may be NULL and k_r, v_r are not read.
+ */
+int augtree_replay_fwd_state(const augtree_plan_t *plan, const void *q_r, const void *k_r, const void *v_r,
+                             const void *k_p, const void *v_p, float *state_o, float *state_lse, int include_own,
+                             void *ws, size_t ws_bytes, void *stream);
+int augtree_merge_states(const augtree_plan_t *plan, int n_states, const float *const *state_o,
+                         const float *const *state_lse, void *o_r, float *lse_r, void *stream);
+int augtree_replay_bwd_state(const augtree_plan_t *plan, const void *q_r, const void *k_r, const void *v_r,
+                             const void *k_p, const void *v_p, const void *o_r, const float *lse_r, const void *do_r,
+                             float *dq_part, void *dk_r, void *dv_r, float *dkp_acc, float *dvp_acc, int include_own,
+                             void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Work accounting (no counterpart in the paper's method).  Every tile kernel
  * counts the work items it has finished; the host counts the items it has
  * handed to launches.  Synchronises the plan's device and returns both counts

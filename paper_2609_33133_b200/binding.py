@@ -33,7 +33,8 @@ EXPORTS = ["augtree_plan_create", "augtree_plan_destroy", "augtree_plan_workspac
            "augtree_prefill_fwd", "augtree_replay_fwd", "augtree_replay_bwd", "augtree_prefill_bwd",
            "augtree_last_device_status", "augtree_launch_count", "augtree_status_string",
            "augtree_set_timing", "augtree_get_kernel_time", "augtree_replay_fwd_static", "augtree_assign_grid",
-           "augtree_items_completed", "augtree_plan_tree"]
+           "augtree_items_completed", "augtree_plan_tree", "augtree_replay_fwd_state", "augtree_merge_states",
+           "augtree_replay_bwd_state"]
 
 
 class Desc(C.Structure):
@@ -55,6 +56,9 @@ lib.augtree_replay_fwd.argtypes = [_vp] + [_vp] * 7 + [_vp, _sz, _vp]
 lib.augtree_replay_fwd_static.argtypes = [_vp] + [_vp] * 7 + [_vp]
 lib.augtree_replay_bwd.argtypes = [_vp] + [_vp] * 13 + [_vp, _sz, _vp]
 lib.augtree_prefill_bwd.argtypes = [_vp] + [_vp] * 11 + [_vp, _sz, _vp]
+lib.augtree_replay_fwd_state.argtypes = [_vp] + [_vp] * 7 + [C.c_int, _vp, _sz, _vp]
+lib.augtree_merge_states.argtypes = [_vp, C.c_int, C.POINTER(_vp), C.POINTER(_vp), _vp, _vp, _vp]
+lib.augtree_replay_bwd_state.argtypes = [_vp] + [_vp] * 13 + [C.c_int, _vp, _sz, _vp]
 lib.augtree_last_device_status.argtypes = [_vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
 lib.augtree_set_timing.argtypes = [_vp, C.c_int]
 lib.augtree_get_kernel_time.argtypes = [_vp, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_int)]
@@ -192,6 +196,24 @@ class Plan:
         for callers that cannot allocate a workspace.  Calls on one device share that array."""
         _check(lib.augtree_replay_fwd_static(self._h, _ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(k_p), _ptr(v_p), _ptr(o_r),
                                              _ptr(lse_r), self._stream()), "replay_fwd_static")
+
+    def replay_fwd_state(self, q_r, k_r, v_r, k_p, v_p, state_o, state_lse, include_own, ws):
+        """Partial softmax state of every response query over this plan's prompt keys (+ its own causal prefix)."""
+        _check(lib.augtree_replay_fwd_state(self._h, _ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(k_p), _ptr(v_p), _ptr(state_o),
+                                            _ptr(state_lse), int(bool(include_own)), _ptr(ws), ws.numel() * ws.element_size(),
+                                            self._stream()), "replay_fwd_state")
+
+    def merge_states(self, states_o, states_lse, o_r, lse_r):
+        n = len(states_o)
+        po = (C.c_void_p * n)(*[t.data_ptr() for t in states_o])
+        pl = (C.c_void_p * n)(*[t.data_ptr() for t in states_lse])
+        _check(lib.augtree_merge_states(self._h, n, po, pl, _ptr(o_r), _ptr(lse_r), self._stream()), "merge_states")
+
+    def replay_bwd_state(self, q_r, k_r, v_r, k_p, v_p, o_r, lse_r, do_r, dq_part, dk_r, dv_r, dkp_acc, dvp_acc, include_own, ws):
+        _check(lib.augtree_replay_bwd_state(self._h, _ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(k_p), _ptr(v_p), _ptr(o_r), _ptr(lse_r),
+                                            _ptr(do_r), _ptr(dq_part), _ptr(dk_r), _ptr(dv_r), _ptr(dkp_acc), _ptr(dvp_acc),
+                                            int(bool(include_own)), _ptr(ws), ws.numel() * ws.element_size(), self._stream()),
+               "replay_bwd_state")
 
     def replay_bwd(self, q_r, k_r, v_r, k_p, v_p, o_r, lse_r, do_r, dq_r, dk_r, dv_r, dkp_acc, dvp_acc, ws):
         _check(lib.augtree_replay_bwd(self._h, _ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(k_p), _ptr(v_p), _ptr(o_r),

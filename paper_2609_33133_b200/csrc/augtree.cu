@@ -102,7 +102,7 @@ long long wait_budget(const augtree_plan *pl) {
 template <int D>
 int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long q_tok, const void *ka, const void *va,
                long long a_tok, const void *kb, const void *vb, long long b_tok, void *o, float *lse, float *part_o,
-               float *part_lse, void *ws, cudaStream_t st) {
+               float *part_lse, void *ws, cudaStream_t st, int state_mode = 0) {
   if (s.n_items() == 0) return AUGTREE_OK;
   // first 256 bytes of the scratch: largest squared key norm per KV head (score bound of the tile kernel)
   unsigned int *kmax2 = static_cast<unsigned int *>(ws);
@@ -131,6 +131,7 @@ int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long 
   const int kind = (int)(&s - pl->sched);
   p.wait_budget = wait_budget(pl); p.kind = kind;
   p.test_flags = (pl->flags & AUGTREE_FLAG_TEST_SKIP_FWD_LOAD) ? TEST_SKIP_FWD_LOAD : 0;
+  p.state_mode = state_mode;
   pl->launched_items[kind] += s.n_items();
   timing_mark(pl, kind, false, st);
   fwd_kernel<D><<<pl->n_lanes, kFwdThreads, FwdSmem<D>::kBytes, st>>>(mq, mka, mva, mkb, mvb, p);
@@ -154,6 +155,8 @@ struct BwdArgs {
   const Sched *dq_sched;   // query-side units
   // key ranges of the query-side kernel: unmasked range tensor (a), causal range tensor (b)
   const void *ka, *va; long long a_tok;
+  int no_own = 0;           // partial-state variant: only the plan's prompt keys (mode-1 items, no causal range in dQ)
+  float *dq_f32 = nullptr;  // partial-state variant: fp32 dQ contribution
 };
 
 // One backward call: row statistics, then the key-side kernel (dK, dV), then the query-side kernel (dQ).
@@ -185,7 +188,13 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     const int kind = (int)(&s - pl->sched);
     p.wait_budget = wait_budget(pl); p.kind = kind;
     p.test_flags = (pl->flags & AUGTREE_FLAG_TEST_SKIP_BWD_LOAD) ? TEST_SKIP_BWD_LOAD : 0;
-    pl->launched_items[kind] += s.n_items();
+    p.no_own = a.no_own;
+    long long n_run = s.n_items();
+    if (a.no_own) {
+      n_run = 0;
+      for (int i = 0; i < s.n_items(); ++i) n_run += s.items[(size_t)i * s.item_ints + 4] != 0;
+    }
+    pl->launched_items[kind] += n_run;
     timing_mark(pl, kind, false, st);
     bwd_kernel<D><<<pl->n_lanes, kBwdThreads, BwdSmem<D>::kBytes, st>>>(mq, mdo, mk0, mv0, mk1, mv1, p);
     timing_mark(pl, kind, true, st);
@@ -202,6 +211,7 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     p.scale = pl->scale; p.scale_log2 = pl->scale * 1.4426950408889634f; p.status = pl->d_status;
     const int kind = (int)(a.dq_sched - pl->sched);
     p.wait_budget = wait_budget(pl); p.kind = kind;
+    p.no_own = a.no_own; p.dq_f32 = a.dq_f32;
     pl->launched_items[kind] += a.dq_sched->n_items();
     timing_mark(pl, kind, false, st);
     // causal keys come from the queries' own sequence tensor (k0/v0)
@@ -442,6 +452,78 @@ int augtree_replay_fwd_static(const augtree_plan_t *pl, const void *q_r, const v
     scratch = g_static_ptr[pl->device];
   }
   return augtree_replay_fwd(pl, q_r, k_r, v_r, k_p, v_p, o_r, lse_r, scratch, AUGTREE_STATIC_SCRATCH_BYTES, stream);
+}
+
+int augtree_replay_fwd_state(const augtree_plan_t *pl, const void *q_r, const void *k_r, const void *v_r, const void *k_p,
+                             const void *v_p, float *state_o, float *state_lse, int include_own, void *ws, size_t ws_bytes,
+                             void *stream) {
+  int r = check_plan(pl);
+  if (r) return r;
+  if (pl->max_splits != 1) return AUGTREE_ERR_UNSUPPORTED;   // a state is one shard's: the plan itself must not shard again
+  if (pl->total_r == 0) return AUGTREE_OK;
+  if (!q_r || !k_r || !v_r || !k_p || !v_p || !state_o || !state_lse) return AUGTREE_ERR_INVALID_ARG;
+  if (!aligned16(q_r) || !aligned16(k_r) || !aligned16(v_r) || !aligned16(k_p) || !aligned16(v_p) || !aligned16(state_o))
+    return AUGTREE_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < pl->ws_fwd || !aligned16(ws)) return AUGTREE_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Sched &s = pl->sched[SCHED_REPLAY_FWD];
+  const int mode = STATE_OUT | (include_own ? 0 : STATE_NO_OWN);
+  if (pl->head_dim == 128)
+    return launch_fwd<128>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, nullptr, nullptr, state_o, state_lse, ws, st, mode);
+  return launch_fwd<64>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, nullptr, nullptr, state_o, state_lse, ws, st, mode);
+}
+
+int augtree_merge_states(const augtree_plan_t *pl, int n_states, const float *const *state_o, const float *const *state_lse,
+                         void *o_r, float *lse_r, void *stream) {
+  int r = check_plan(pl);
+  if (r) return r;
+  if (n_states < 1 || n_states > kMaxStates || !state_o || !state_lse || !o_r || !lse_r) return AUGTREE_ERR_INVALID_ARG;
+  if (pl->total_r == 0) return AUGTREE_OK;
+  StatePtrs sp;
+  sp.n = n_states;
+  for (int i = 0; i < n_states; ++i) {
+    if (!state_o[i] || !state_lse[i]) return AUGTREE_ERR_INVALID_ARG;
+    sp.o[i] = state_o[i]; sp.lse[i] = state_lse[i];
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const long long warps = pl->total_r * (long long)pl->h_q;
+  const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
+  if (pl->head_dim == 128)
+    merge_states_kernel<128><<<blocks, 256, 0, st>>>(sp, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q);
+  else
+    merge_states_kernel<64><<<blocks, 256, 0, st>>>(sp, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q);
+  ++g_launches;
+  return cudaGetLastError() == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+}
+
+int augtree_replay_bwd_state(const augtree_plan_t *pl, const void *q_r, const void *k_r, const void *v_r, const void *k_p,
+                             const void *v_p, const void *o_r, const float *lse_r, const void *do_r, float *dq_part, void *dk_r,
+                             void *dv_r, float *dkp_acc, float *dvp_acc, int include_own, void *ws, size_t ws_bytes, void *stream) {
+  int r = check_plan(pl);
+  if (r) return r;
+  if (!dkp_acc || !dvp_acc) return AUGTREE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (pl->flags & AUGTREE_FLAG_ZERO_PROMPT_GRAD) {
+    const size_t bytes = (size_t)pl->total_p * pl->h_kv * pl->head_dim * 4;
+    if (cudaMemsetAsync(dkp_acc, 0, bytes, st) != cudaSuccess || cudaMemsetAsync(dvp_acc, 0, bytes, st) != cudaSuccess)
+      return AUGTREE_ERR_CUDA;
+  }
+  if (pl->total_r == 0) return AUGTREE_OK;
+  if (!q_r || !k_r || !v_r || !k_p || !v_p || !o_r || !lse_r || !do_r || !dq_part) return AUGTREE_ERR_INVALID_ARG;
+  if (include_own && (!dk_r || !dv_r)) return AUGTREE_ERR_INVALID_ARG;
+  if (!aligned16(q_r) || !aligned16(k_r) || !aligned16(v_r) || !aligned16(k_p) || !aligned16(v_p) || !aligned16(o_r) ||
+      !aligned16(do_r) || !aligned16(dq_part) || !aligned16(dk_r) || !aligned16(dv_r) || !aligned16(dkp_acc) || !aligned16(dvp_acc))
+    return AUGTREE_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < pl->ws_bwd || !aligned16(ws)) return AUGTREE_ERR_WORKSPACE;
+  BwdArgs a;
+  a.q = q_r; a.d_o = do_r; a.o = o_r; a.lse = lse_r; a.q_tok = pl->total_r;
+  a.k0 = k_r; a.v0 = v_r; a.kv0_tok = pl->total_r; a.k1 = k_p; a.v1 = v_p; a.kv1_tok = pl->total_p;
+  a.dq = nullptr; a.dk_out = dk_r; a.dv_out = dv_r; a.dk_acc = dkp_acc; a.dv_acc = dvp_acc; a.causal_fp32 = 0;
+  a.d_segs = pl->d_seg_replay; a.d_tiles = pl->d_tiles_replay; a.n_tiles = (long long)pl->tiles_replay.size() / 2;
+  a.dq_sched = &pl->sched[SCHED_REPLAY_DQ]; a.ka = k_p; a.va = v_p; a.a_tok = pl->total_p;
+  a.no_own = include_own ? 0 : 1; a.dq_f32 = dq_part;
+  const Sched &s = pl->sched[SCHED_REPLAY_BWD];
+  return pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, st) : launch_bwd<64>(pl, s, a, ws, st);
 }
 
 int augtree_replay_bwd(const augtree_plan_t *pl, const void *q_r, const void *k_r, const void *v_r, const void *k_p,

@@ -43,6 +43,7 @@ struct BwdParams {
   long long wait_budget;    // clocks a wait may take before the kernel gives up
   int kind;                 // schedule index: status[2 + kind] counts finished items
   int test_flags;           // TEST_SKIP_BWD_LOAD: lane 0 never loads the first dO tile of its first item
+  int no_own;               // partial-state variant: items inside a sequence (mode 0) are skipped by every role
 };
 
 constexpr int kBwdThreads = 576;  // 16 element-wise warps, TMA warp, MMA warp
@@ -124,9 +125,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       tma_prefetch_desc(&tm_v0); tma_prefetch_desc(&tm_k1); tma_prefetch_desc(&tm_v1);
       uint32_t ic = 0, T = 0;
       bool ok = true;
-      for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
+      for (int it = it_begin; it < it_end && ok; ++it) {
         const int32_t *I = p.items + (size_t)it * 8;
         const int kv_tok0 = I[0], kv_pos0 = I[1], kvh = I[3], mode = I[4], seg0 = I[5], nseg = I[6];
+        if (p.no_own && mode == 0) continue;
         if (ic > 0) {
           ok = mbar_wait(bar_kv_empty, (ic - 1) & 1, ab, WAIT_BWD_KV_EMPTY);
           if (!ok) break;
@@ -156,6 +158,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               for (int b = 0; b < NBOX; ++b) tma_load_3d(sDo0 + st * TILE + b * 16384, &tm_do, bar_do_full + 8 * st, b * 64, head, row);
             }
         }
+        ++ic;
       }
     }
   } else if (warp == 17) {
@@ -178,9 +181,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         tc_fence_after();
         return true;
       };
-      for (int it = it_b; it < it_e && ok; ++it, ++ic) {
+      for (int it = it_b; it < it_e && ok; ++it) {
         const int32_t *I = p.items + (size_t)it * 8;
         const int kv_pos0 = I[1], mode = I[4], seg0 = I[5], nseg = I[6];
+        if (p.no_own && __shfl_sync(0xffffffffu, mode, 0) == 0) continue;
         int n_pairs = 0;
         for (int sg = seg0; sg < seg0 + nseg; ++sg) {
           const int nqt = (p.segs[3 * sg + 1] + 127) >> 7;
@@ -251,6 +255,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
         if (!ok) break;
         if (elected) { tc_commit(bar_acc_full); tc_commit(bar_kv_empty); }
+        ++ic;
       }
     }
   } else {
@@ -307,9 +312,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       return true;
     };
 
-    for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
+    for (int it = it_begin; it < it_end && ok; ++it) {
       const int32_t *I = p.items + (size_t)it * 8;
       const int kv_tok0 = I[0], kv_pos0 = I[1], kv_rows = I[2], kvh = I[3], mode = I[4], seg0 = I[5], nseg = I[6];
+      if (p.no_own && mode == 0) continue;
       const bool key_valid = r < kv_rows;
       bool first = true;
       for (int sg = seg0; sg < seg0 + nseg && ok; ++sg) {
@@ -405,6 +411,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       tc_fence_before();
       warp_arrive(bar_acc_empty);
       if (warp == 0 && lane == 0) atomicAdd(p.status + 2 + p.kind, 1);  // item finished (work accounting)
+      ++ic;
     }
   }
 

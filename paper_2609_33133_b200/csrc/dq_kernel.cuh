@@ -35,6 +35,8 @@ struct DqParams {
   int *status;
   long long wait_budget;    // clocks a wait may take before the kernel gives up
   int kind;                 // schedule index: status[2 + kind] counts finished items
+  int no_own;               // partial-state variant: the causal range of the query's own sequence is left out
+  float *dq_f32;            // partial-state variant: dQ is written here in fp32 (summed over KV owners afterwards)
 };
 
 constexpr int kDqThreads = 320;
@@ -112,7 +114,8 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       bool ok = true;
       for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
         const int32_t *I = p.items + (size_t)it * 12;
-        const int q_tok0 = I[0], head = I[3], a_tok0 = I[4], a_len = I[5], b_tok0 = I[6], b_len = I[7], tile = I[8], kvh = I[11];
+        const int q_tok0 = I[0], head = I[3], a_tok0 = I[4], a_len = I[5], b_tok0 = I[6], tile = I[8], kvh = I[11];
+        const int b_len = p.no_own ? 0 : I[7];
         const int nA = (a_len + 127) >> 7, n = nA + ((b_len + 127) >> 7);
         ok = mbar_wait(bar_qdo_empty, (ic & 1) ^ 1, ab, WAIT_DQ_QDO);
         if (!ok) break;
@@ -175,7 +178,7 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       };
       for (int it = it_b; it < it_e && ok; ++it, ++ic) {
         const int32_t *I = p.items + (size_t)it * 12;
-        const int n = __shfl_sync(0xffffffffu, ((I[5] + 127) >> 7) + ((I[7] + 127) >> 7), 0);
+        const int n = __shfl_sync(0xffffffffu, ((I[5] + 127) >> 7) + (p.no_own ? 0 : ((I[7] + 127) >> 7)), 0);
         ok = mbar_wait(bar_qt_ready, ic & 1, ab, WAIT_DQ_QT);
         if (!ok) break;
         bool have_sread = false, have_ds = false, have_v = false, have_k = false;
@@ -226,7 +229,8 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     bool ok = true;
     for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
       const int32_t *I = p.items + (size_t)it * 12;
-      const int q_tok0 = I[0], q_pos0 = I[1], q_rows = I[2], head = I[3], a_len = I[5], b_len = I[7];
+      const int q_tok0 = I[0], q_pos0 = I[1], q_rows = I[2], head = I[3], a_len = I[5];
+      const int b_len = p.no_own ? 0 : I[7];
       const int nA = (a_len + 127) >> 7, n = nA + ((b_len + 127) >> 7);
       // ---- Q and dO rows into TMEM as bf16 A operands; this thread: row r, columns (D/2)*ch .. of d
       ok = mbar_wait(bar_qdo_full, ic & 1, ab, WAIT_DQ_QDO);
@@ -323,7 +327,12 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           uint32_t v[32];
           tmem_ld32(tDQ + lane_off + ch * HALF + c * 32, v);
           tc_wait_ld();
-          if (r < q_rows) {
+          if (r < q_rows && p.dq_f32) {
+            float4 *dst = reinterpret_cast<float4 *>(p.dq_f32 + (((long long)q_tok0 + r) * p.h_q + head) * D + ch * HALF + c * 32);
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              dst[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]), __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
+          } else if (r < q_rows) {
             uint4 *dst = reinterpret_cast<uint4 *>(dst_row + c * 32);
 #pragma unroll
             for (int e = 0; e < 4; ++e)

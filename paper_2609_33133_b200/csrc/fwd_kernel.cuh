@@ -37,7 +37,14 @@ struct FwdParams {
   long long wait_budget;    // clocks a wait may take before the kernel gives up
   int kind;                 // schedule index: status[2 + kind] counts finished items
   int test_flags;           // TEST_SKIP_FWD_LOAD: lane 0 never loads the first V tile of its first item
+  int state_mode;           // STATE_OUT | STATE_NO_OWN: partial-state variant for context-parallel replay (below)
 };
+
+// Partial-state variant (Sec. 3.3, "Common tile semantics": a query block against one KV shard gives a partial
+// state; the states along a query's row are merged afterwards).  STATE_OUT: every item writes its normalised fp32
+// output and its LSE into part_o / part_lse (shard slot 0) instead of the final tensors.  STATE_NO_OWN: the causal
+// range of the query's own sequence is left out, so that the state covers the plan's prompt keys alone.
+enum : int { STATE_OUT = 1, STATE_NO_OWN = 2 };
 
 constexpr int kFwdThreads = 320;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: P stays <= 2^8 while the row maximum is tracked
@@ -125,7 +132,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       bool ok = true;
       for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
         const int32_t *I = p.items + (size_t)it * 12;
-        const int q_tok0 = I[0], head = I[3], a_tok0 = I[4], a_len = I[5], b_tok0 = I[6], b_len = I[7], kvh = I[11];
+        const int q_tok0 = I[0], head = I[3], a_tok0 = I[4], a_len = I[5], b_tok0 = I[6], kvh = I[11];
+        const int b_len = (p.state_mode & STATE_NO_OWN) ? 0 : I[7];
         const int nA = (a_len + 127) >> 7, n = nA + ((b_len + 127) >> 7);
         ok = mbar_wait(bar_q_empty, (ic & 1) ^ 1, ab, WAIT_FWD_Q_EMPTY);
         if (!ok) break;
@@ -193,7 +201,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       };
       for (int it = it_b; it < it_e && ok; ++it, ++ic) {
         const int32_t *I = p.items + (size_t)it * 12;
-        const int n = __shfl_sync(0xffffffffu, ((I[5] + 127) >> 7) + ((I[7] + 127) >> 7), 0);
+        const int n = __shfl_sync(0xffffffffu, ((I[5] + 127) >> 7) + ((p.state_mode & STATE_NO_OWN) ? 0 : ((I[7] + 127) >> 7)), 0);
         ok = mbar_wait(bar_q_full, ic & 1, ab, WAIT_FWD_Q_FULL);
         if (!ok) break;
         bool have_p0 = false;
@@ -305,8 +313,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #endif
     for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
       const int32_t *I = p.items + (size_t)it * 12;
-      const int q_tok0 = I[0], q_pos0 = I[1], q_rows = I[2], head = I[3], a_len = I[5], b_len = I[7];
-      const int split = I[8], n_splits = I[9];
+      const int q_tok0 = I[0], q_pos0 = I[1], q_rows = I[2], head = I[3], a_len = I[5];
+      const int b_len = (p.state_mode & STATE_NO_OWN) ? 0 : I[7];
+      const int split = (p.state_mode & STATE_OUT) ? 0 : I[8], n_splits = (p.state_mode & STATE_OUT) ? 2 : I[9];
       const int nA = (a_len + 127) >> 7, n = nA + ((b_len + 127) >> 7);
       // per unit u and row (A, B): running reference maximum and this thread's share of the row sum
       float mA[2] = {0.f, 0.f}, mB[2] = {0.f, 0.f}, lA[2] = {0.f, 0.f}, lB[2] = {0.f, 0.f};
@@ -529,6 +538,45 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   tc_fence_before();
   __syncthreads();
   if (warp == 9) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+}
+
+// Merge of up to kMaxStates partial states that live in separate buffers (one per KV shard owner: the states a
+// query's owner receives in MoveQ, Sec. 3.3): one warp per (token, head);
+// LSE = log sum_s exp(lse_s), O = sum_s exp(lse_s - LSE) O_s.  A shard that saw no key has lse = -inf and weight 0.
+constexpr int kMaxStates = 16;
+struct StatePtrs {
+  const float *o[kMaxStates];    // [tokens, h_q, D] fp32, normalised
+  const float *lse[kMaxStates];  // [h_q, tokens]
+  int n;
+};
+template <int D>
+__global__ void merge_states_kernel(const StatePtrs sp, __nv_bfloat16 *o, float *lse, long long n_tok, int h_q) {
+  const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= n_tok * h_q) return;
+  const long long tok = w / h_q;
+  const int head = (int)(w % h_q);
+  float mx = -INFINITY;
+  for (int s = 0; s < sp.n; ++s) mx = fmaxf(mx, sp.lse[s][(long long)head * n_tok + tok]);
+  const float ref = mx == -INFINITY ? 0.f : mx;
+  float den = 0.f;
+  for (int s = 0; s < sp.n; ++s) den += __expf(sp.lse[s][(long long)head * n_tok + tok] - ref);
+  constexpr int PER = D / 32;
+  float acc[PER];
+#pragma unroll
+  for (int i = 0; i < PER; ++i) acc[i] = 0.f;
+  for (int s = 0; s < sp.n; ++s) {
+    const float wgt = __expf(sp.lse[s][(long long)head * n_tok + tok] - ref) / den;
+    const float *src = sp.o[s] + (tok * h_q + head) * D + lane * PER;
+    if (wgt > 0.f) {
+#pragma unroll
+      for (int i = 0; i < PER; ++i) acc[i] += wgt * src[i];
+    }
+  }
+  __nv_bfloat16 *dst = o + (tok * h_q + head) * D + lane * PER;
+#pragma unroll
+  for (int i = 0; i < PER; ++i) dst[i] = __float2bfloat16(acc[i]);
+  if (lane == 0) lse[(long long)head * n_tok + tok] = ref + __logf(den);
 }
 
 // Largest squared key norm per KV head over the K tensors of one forward call (the unmasked-range tensor and,
