@@ -1,4 +1,6 @@
-"""MoveQ, the KV-stationary replay primitive of Sec. 3.3, on top of the library's partial-state entry points.
+"""The two replay primitives of Sec. 3.3, MoveQ and TreeMoveKV, on top of the library's partial-state entry points.
+
+MoveQ first; TreeMoveKV (lane-local KV rings under a replay-grid placement) at the end of the file.
 
 Rank r of n keeps shard r of every group's prompt KV (stationary) and owns some response branches (their K/V,
 their queries, their outputs).  Forward: the response queries of all branches are made known to every rank, each
@@ -215,3 +217,84 @@ def moveq_rank(dist, backend, w, rank: int, world: int, local: Dict[str, torch.T
         mine[torch.as_tensor(_rows(lay, lay.owned), device=q_all.device)] = True
     keep = lambda x, rows_first=True: x * (mine[:, None, None] if rows_first else mine[None, :]).to(x.dtype)
     return {"o_r": keep(o_all), "lse_r": keep(lse_all, False), "dq_r": keep(dq_part), "dk_r": dk_r, "dv_r": dv_r, "dk_p": dkp, "dv_p": dvp}
+
+
+# --------------------------------------------------------------------------------------------------------------
+# TreeMoveKV (Sec. 3.3): response-local move-KV.  The d ranks form s lanes of d_lane = d / s ranks; a placement X
+# (Eq. 6, augtree_assign_grid) gives every response path a (round, lane) cell; a lane keeps the whole prompt KV,
+# sharded over its d_lane ranks, and within a round each of its ranks owns some of the cell's paths whole (queries,
+# response K/V and outputs never leave their rank: response-path locality).  Only the prompt-KV shards travel: in
+# ring stage t rank r holds shard (r - t) mod d_lane, computes the partial state of its own queries over it and
+# merges it into their running state; in the backward pass the shards go round once more with their fp32 dK_P / dV_P
+# accumulators, every rank adds its queries' share (Eq. 2 accumulated along the ring) and keeps its dQ to itself.
+def treemovekv_emulate(binding, w, t, s: int, d_lane: int, rounds: int = 1, device=0):
+    """All ranks of a TreeMoveKV replay (s lanes x d_lane ranks, `rounds` rounds) in one process on one GPU, stage by
+    stage.  One group only (a replay tree).  Returns the same tensors as moveq_emulate plus the placement used."""
+    if w.n_groups != 1 or d_lane > 16:
+        raise ValueError("one replay tree at a time, lanes of at most 16 ranks")
+    P, R = w.prompt_len[0], w.branch_len[0]
+    tiles = lambda r: -(-r // 128) * -(-P // 128) + (-(-r // 128)) * (-(-r // 128) + 1) // 2   # unit weight: valid tile count
+    x_round, x_lane, _, _ = binding.assign_grid([tiles(r) for r in R], R, n_rounds=rounds, n_lanes=s)
+    bounds = shard_bounds(P, d_lane)
+    cu_r = np.concatenate([[0], np.cumsum(R)]).astype(np.int64)
+    hq, hkv, d = w.h_q, w.h_kv, w.head_dim
+    dev = "cuda"
+    kp = [t["k_p"][a:b].contiguous() for a, b in bounds]
+    vp = [t["v_p"][a:b].contiguous() for a, b in bounds]
+    out = {"o_r": torch.zeros((w.total_response, hq, d), device=dev, dtype=torch.bfloat16),
+           "lse_r": torch.zeros((hq, w.total_response), device=dev, dtype=torch.float32),
+           "dq_r": torch.zeros((w.total_response, hq, d), device=dev, dtype=torch.float32),
+           "dk_r": torch.zeros((w.total_response, hkv, d), device=dev, dtype=torch.bfloat16),
+           "dv_r": torch.zeros((w.total_response, hkv, d), device=dev, dtype=torch.bfloat16),
+           "dk_p": torch.zeros((P, hkv, d), device=dev, dtype=torch.float32),
+           "dv_p": torch.zeros((P, hkv, d), device=dev, dtype=torch.float32)}
+    plans = []
+    for rnd in range(rounds):
+        for lane in range(s):
+            cell = [k for k in range(len(R)) if x_round[k] == rnd and x_lane[k] == lane]
+            # every lane holds its own copy of the prompt-KV shards, and so its own accumulators for them
+            acc = [(torch.zeros((b - a, hkv, d), device=dev, dtype=torch.float32), torch.zeros((b - a, hkv, d), device=dev, dtype=torch.float32))
+                   for a, b in bounds]
+            for r in range(d_lane):
+                mine = [k for i, k in enumerate(cell) if i % d_lane == r]
+                if not mine:
+                    continue
+                rows = torch.as_tensor(np.concatenate([np.arange(cu_r[k], cu_r[k + 1]) for k in mine]), device=dev)
+                sel = lambda x: x.index_select(0, rows).contiguous()
+                q, k_r, v_r, do = sel(t["q_r"]), sel(t["k_r"]), sel(t["v_r"]), sel(t["do_r"])
+                stage_plans = [binding.Plan([b - a], [[R[k] for k in mine]], hq, hkv, d, device=device) for a, b in bounds]
+                plans += stage_plans
+                ws = torch.empty(max(max(p.ws_fwd_bytes, p.ws_bwd_bytes) for p in stage_plans) + 256, device=dev, dtype=torch.uint8)
+                n = int(rows.numel())
+                # forward ring: one partial state per stage (stage 0: the rank's own shard and the paths' own causal
+                # prefixes); the merge is associative, so the d_lane states are folded once, after the last stage
+                states_o, states_l = [], []
+                for stage in range(d_lane):
+                    j = (r - stage) % d_lane
+                    so = torch.empty((n, hq, d), device=dev, dtype=torch.float32)
+                    sl = torch.empty((hq, n), device=dev, dtype=torch.float32)
+                    stage_plans[j].replay_fwd_state(q, k_r, v_r, kp[j], vp[j], so, sl, stage == 0, ws)
+                    states_o.append(so); states_l.append(sl)
+                o = torch.empty((n, hq, d), device=dev, dtype=torch.bfloat16)
+                lse = torch.empty((hq, n), device=dev, dtype=torch.float32)
+                stage_plans[0].merge_states(states_o, states_l, o, lse)
+                # backward ring: shards come round again with their accumulators
+                dq = torch.zeros((n, hq, d), device=dev, dtype=torch.float32)
+                dk = torch.empty((n, hkv, d), device=dev, dtype=torch.bfloat16)
+                dv = torch.empty_like(dk)
+                for stage in range(d_lane):
+                    j = (r - stage) % d_lane
+                    part = torch.empty((n, hq, d), device=dev, dtype=torch.float32)
+                    stage_plans[j].replay_bwd_state(q, k_r, v_r, kp[j], vp[j], o, lse, do, part, dk, dv, acc[j][0], acc[j][1], stage == 0, ws)
+                    dq += part
+                out["o_r"][rows], out["dq_r"][rows], out["dk_r"][rows], out["dv_r"][rows] = o, dq, dk, dv
+                out["lse_r"][:, rows] = lse
+            # the lanes' copies of the prompt-KV gradient are summed when the prefill graphs are joined (Eq. 2 over lanes)
+            for (a, b), (gk, gv) in zip(bounds, acc):
+                out["dk_p"][a:b] += gk
+                out["dv_p"][a:b] += gv
+    torch.cuda.synchronize()
+    if any(p.device_status() != (0, 0) for p in plans):
+        raise RuntimeError("device status")
+    out["placement"] = (x_round, x_lane)
+    return out

@@ -57,3 +57,26 @@ def test_moveq_emulation_matches_oracle(B, case, world):
         one = cp.moveq_emulate(B, w, t, 1)
         assert np.array_equal(f64(one["lse_r"]), whole["lse_r"])
         assert np.abs(f64(one["o_r"]) - whole["o_r"]).max() <= 2.0 ** -7 * np.abs(whole["o_r"]).max()   # fp32 state -> bf16 once more
+
+
+@pytest.mark.parametrize("s_lanes,d_lane,rounds", [(1, 2, 1), (2, 2, 1), (2, 3, 2), (4, 1, 1)])
+def test_treemovekv_emulation_matches_oracle(B, s_lanes, d_lane, rounds):
+    """TreeMoveKV: lanes from the replay-grid placement (Eq. 6), prompt-KV shards going round each lane's ring, the
+    shards' gradient accumulators going round again; every path stays on one rank."""
+    from paper_2609_33133_b200 import cp
+    w = wl.Workload("tmkv", [900], [[300, 150, 420, 64, 257, 130]], 8, 2, 128, 84)
+    t_cpu = wl.make_tensors(w)
+    t = {k: v.cuda() for k, v in t_cpu.items()}
+    res = cp.treemovekv_emulate(B, w, t, s_lanes, d_lane, rounds)
+    x_round, x_lane = res.pop("placement")
+    assert max(x_round) < rounds and max(x_lane) < s_lanes and len(x_lane) == 6
+    plan = B.Plan(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, device=0)
+    out = B.alloc_outputs(plan)
+    out["dk_p"].copy_(res["dk_p"]); out["dv_p"].copy_(res["dv_p"])
+    plan.prefill_fwd(t["q_p"], t["k_p"], t["v_p"], out["o_p"], out["lse_p"], out["ws"])
+    plan.prefill_bwd(t["q_p"], t["k_p"], t["v_p"], out["o_p"], out["lse_p"], t["do_p"], out["dk_p"], out["dv_p"], out["dq_p"], None, None, out["ws"])
+    torch.cuda.synchronize()
+    f64 = lambda x: x.float().cpu().numpy().astype(np.float64)
+    got = {k: f64(res[k]) for k in ("o_r", "lse_r", "dq_r", "dk_r", "dv_r")}
+    got.update({k: f64(out[k]) for k in ("o_p", "lse_p", "dq_p", "dk_p", "dv_p")})
+    pu.assert_parity_elementwise(got, pu.run_oracle(w, t_cpu), pu.rounding_error_sigma(w, t_cpu))
