@@ -654,14 +654,6 @@ int augtree_get_kernel_time(const augtree_plan_t *pl, int kernel, float *total_m
 
 long long augtree_launch_count(void) { return g_launches.load(); }
 
-#if AUGTREE_TRACE
-// Measurement build only (not declared in the public header): reads and clears the forward kernel's phase counters.
-int augtree_debug_fwd_trace(unsigned long long *out8) {
-  unsigned long long z[8] = {};
-  if (cudaMemcpyFromSymbol(out8, g_fwd_trace, sizeof(z)) != cudaSuccess) return AUGTREE_ERR_CUDA;
-  return cudaMemcpyToSymbol(g_fwd_trace, z, sizeof(z)) == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
-}
-#endif
 
 const char *augtree_status_string(int s) {
   switch (s) {

@@ -53,22 +53,10 @@ constexpr float kRescaleThreshold = 8.0f;  // log2 units: P stays <= 2^8 while t
 // accumulators and bf16's fp32-sized exponent nothing overflows and nothing loses precision (softmax does not
 // depend on the reference), so the row maximum of the later tiles is not computed at all.
 constexpr float kSkipMaxHeadroom = 60.0f;
-#ifndef AUGTREE_FWD_SPLIT_WG
-#define AUGTREE_FWD_SPLIT_WG 0
-#endif
 #ifndef AUGTREE_FWD_FMA_MASK
 #define AUGTREE_FWD_FMA_MASK 0x8888u
 #endif
 constexpr uint32_t kFwdFmaMask = AUGTREE_FWD_FMA_MASK;  // column blocks (of 16) whose exp2 runs on the FMA pipe
-
-#if AUGTREE_TRACE
-// Measurement build only: clock64 spans of the softmax phases, summed over warp 1 of every CTA
-// (0 wait for S, 1 TMEM load, 6 maxima, 7 quad shuffles, 2 rescale test, 3 exponentials, 4 store + hand-off; 5 = passes).
-__device__ unsigned long long g_fwd_trace[8];
-#define TRACE_MARK(k) do { const long long t_ = clock64(); tr[k] += t_ - t_prev; t_prev = t_; } while (0)
-#else
-#define TRACE_MARK(k) do { } while (0)
-#endif
 
 template <int D>
 struct FwdSmem {
@@ -291,13 +279,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // columns the two columns 2 (t % 4), 2 (t % 4) + 1.  A row lives in one quad, so its maximum and sum are
     // two shuffles and no warp waits for another.
     const int cq = 2 * (lane & 3);                         // first of this thread's two columns in a block of 8
-#if AUGTREE_FWD_SPLIT_WG
-    // warps 0-3 own query tile 0, warps 4-7 query tile 1; a warp does its 32 rows as two blocks of 16 (u = 0, 1)
-#define FWD_UNIT(u) const int g = warp >> 2, lane_base = (warp & 3) * 32 + (u) * 16
-#else
     // all eight warps work on query tile u = 0, then on tile 1; a warp does 16 rows of each
 #define FWD_UNIT(u) const int g = (u), lane_base = (warp & 3) * 32 + (warp >> 2) * 16
-#endif
     auto quad_max = [](float x) {
       x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 1));
       return fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 2));
@@ -308,9 +291,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     };
     uint32_t ic = 0, T = 0;
     bool ok = true;
-#if AUGTREE_TRACE
-    long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0}, t_prev = clock64();
-#endif
     for (int it = it_begin; it < it_end && ok; ++it, ++ic) {
       const int32_t *I = p.items + (size_t)it * 12;
       const int q_tok0 = I[0], q_pos0 = I[1], q_rows = I[2], head = I[3], a_len = I[5];
@@ -363,17 +343,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           const int rA = lane_base + (lane >> 2), rB = rA + 8;   // rows inside the query tile
           const uint32_t lane_off = (uint32_t)lane_base << 16;
           const uint32_t tS = tmem + lane_off + g * 128, tO = tmem + lane_off + 256 + g * 128;
-#if AUGTREE_TRACE
-          t_prev = clock64();
-#endif
           ok = mbar_wait(bar_s_full + 8 * g, T & 1, ab, WAIT_FWD_S_FULL);
           if (!ok) break;
           tc_fence_after();
-          TRACE_MARK(0);
           uint32_t s[64];
           tmem_ld_16x256b_x16(tS, s);
           tc_wait_ld();
-          TRACE_MARK(1);
           // number of leading key columns of this KV tile that rows A and B see
           const int lim0 = (j < nA) ? (a_len - j * 128) : (q_pos0 + g * 128 + 1 - (j - nA) * 128);
           const int limA = (j < nA) ? lim0 : lim0 + rA, limB = (j < nA) ? lim0 : lim0 + rB;
@@ -402,10 +377,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               xA = fmaxf(a0, a1);
               xB = fmaxf(b0, b1);
             }
-            TRACE_MARK(6);
             xA = quad_max(xA) * p.scale_log2;
             xB = quad_max(xB) * p.scale_log2;
-            TRACE_MARK(7);
             if (j == 0) {
               mA[u] = (xA == -INFINITY) ? 0.f : xA;
               mB[u] = (xB == -INFINITY) ? 0.f : xB;
@@ -436,7 +409,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               }
             }
           }
-          TRACE_MARK(2);
           // P = exp2(s * scale - m), bf16 pairs in the 16x128b layout over the S columns [0, 64).  The scale-and-
           // subtract, the row sums and the polynomial exponentials run on register pairs (packed fp32: half the
           // issue slots); kFwdFmaMask says which of the 16 column blocks take their exponentials on the FMA
@@ -458,17 +430,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             pk[2 * i + 1] = pack_bf16(pb.x, pb.y);
           }
           const float sA = accA.x + accA.y, sB = accB.x + accB.y;
-          TRACE_MARK(3);
           tmem_st_16x128b_x16(tS, pk);
           lA[u] += sA;
           lB[u] += sB;
           tc_wait_st();
           tc_fence_before();
           warp_arrive(bar_p_full + 8 * g);
-          TRACE_MARK(4);
-#if AUGTREE_TRACE
-          ++tr[5];
-#endif
         }
       }
       if (!ok) break;
@@ -521,10 +488,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       }
       if (ok && warp == 0 && lane == 0) atomicAdd(p.status + 2 + p.kind, 1);  // item finished (work accounting)
     }
-#if AUGTREE_TRACE
-    if (warp == 1 && lane == 0)
-      for (int k = 0; k < 8; ++k) atomicAdd(&g_fwd_trace[k], (unsigned long long)tr[k]);
-#endif
   }
 
   // ---------------------------------------------------------------- teardown
