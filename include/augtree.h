@@ -250,8 +250,9 @@ int augtree_prefill_bwd(const augtree_plan_t *plan, const void *q_p, const void 
  *    call outside any stream capture.
  *  - All calls on a device share the one array and it keeps whatever the last
  *    call left there.  The one part that must start at zero (the key-norm
- *    maxima at its head) is cleared by every call on its stream; every other
- *    value read is written by the same call first.  Two
+ *    maxima at its head, when several blocks combine them) is cleared by the
+ *    call itself on its stream; every other value read is written by the same
+ *    call first.  Two
  *    calls that may overlap on the GPU (different streams, no dependency) race
  *    on it; order them.
  * Arguments and results are those of augtree_replay_fwd.

@@ -544,7 +544,8 @@ __global__ void merge_states_kernel(const StatePtrs sp, __nv_bfloat16 *o, float 
 
 // Largest squared key norm per KV head over the K tensors of one forward call (the unmasked-range tensor and,
 // if different, the causal-range tensor): out[h] = max over tokens of |k[token, h, :]|^2, as the bits of a
-// non-negative float (so an unsigned atomicMax orders them).  `out` is cleared by the caller before the launch.
+// non-negative float (so an unsigned atomicMax orders them).  With more than one block per head `out` is cleared by
+// the caller before the launch; a single block per head (small inputs) stores its result and needs no clearing.
 // Feeds the score bound that lets the tile kernel skip row maxima; HBM-bound, a few microseconds.
 template <int D>
 __global__ void key_norm_kernel(const __nv_bfloat16 *ka, long long a_tok, const __nv_bfloat16 *kb, long long b_tok, int h_kv,
@@ -576,7 +577,14 @@ __global__ void key_norm_kernel(const __nv_bfloat16 *ka, long long a_tok, const 
   }
 #pragma unroll
   for (int sft = 16; sft > 0; sft >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, sft));
-  if (lane == 0) atomicMax(out + head, __float_as_uint(best));
+  __shared__ float warp_best[32];
+  if (lane == 0) warp_best[threadIdx.x >> 5] = best;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < (int)(blockDim.x >> 5); ++i) best = fmaxf(best, warp_best[i]);
+    if (gridDim.x == 1) out[head] = __float_as_uint(best);
+    else atomicMax(out + head, __float_as_uint(best));
+  }
 }
 
 // Merge of the prompt-KV shards' partial states (Sec. 3.3): one warp per

@@ -104,3 +104,24 @@ def test_flop_accounting_matches_oracle_pair_count():
         assert fl["total"] == 14 * w.head_dim * w.h_q * (pre + rep)
         assert abs(fl["reuse_factor"] - flat / (pre + rep)) < 1e-12
     assert abs(bench.useful_flops(wl.config(2))["total"] / 1e12 - 9.2606) < 1e-3
+
+
+def test_bench_records_are_consistent():
+    """Both arms print the same `config` object; the algorithmic bytes of the dominant launch are the sum of the tensors
+    it touches, each crossing once; the tracked ncu table, where present, names the six launches of a step."""
+    import json
+    import os
+    w = wl.config(2)
+    assert bench.config_record(w, 1) == bench.config_record(wl.config(2), 1)
+    # replay key-side backward on configuration 2: Q_R + dO_R 235 MB, statistics 3.7, K/V_R 33.6, K/V_P 16.8, dK_R/dV_R 33.6,
+    # fp32 dK_P/dV_P read + written 67.1
+    q, kv_r, kv_p = 2 * 16384 * 28 * 128, 2 * 16384 * 4 * 128, 2 * 8192 * 4 * 128
+    want = 2 * q + 8 * 16384 * 28 + 2 * kv_r + 2 * kv_p + 2 * kv_r + 2 * 2 * (2 * kv_p)
+    assert bench.algorithmic_bytes(w, "replay_bwd_dkdv") == want and abs(want / 1e9 - 0.39) < 0.005
+    path = os.path.join(os.path.dirname(os.path.abspath(bench.__file__)), "profiles", "ncu_dram_bytes.json")
+    if os.path.exists(path):
+        table = json.load(open(path))
+        for name, rec in table.items():
+            if not name.startswith("_"):
+                assert sorted(rec) == sorted(["prefill_fwd", "replay_fwd", "replay_bwd_dkdv", "replay_bwd_dq", "prefill_bwd_dkdv", "prefill_bwd_dq"])
+                assert bench.ncu_dram_bytes(name, "replay_bwd_dkdv") == rec["replay_bwd_dkdv"] > bench.algorithmic_bytes(wl.config(2), "replay_bwd_dkdv") * 0.5
