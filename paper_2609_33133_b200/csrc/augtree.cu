@@ -110,7 +110,7 @@ int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long 
     const bool same = ka == kb;
     const long long rows = a_tok + (same ? 0 : b_tok);
     // small inputs: one block per head, which stores its maximum (no clearing launch); otherwise clear, then atomicMax
-    const unsigned blocks = rows <= 4096 ? 1u : (unsigned)std::min<long long>(296, rows / 64);
+    const unsigned blocks = rows <= 4096 ? 1u : (unsigned)std::min<long long>(2368, rows / 64);
     if (blocks > 1 && cudaMemsetAsync(kmax2, 0, (size_t)pl->h_kv * sizeof(unsigned int), st) != cudaSuccess) return AUGTREE_ERR_CUDA;
     key_norm_kernel<D><<<dim3(blocks, (unsigned)pl->h_kv), 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(ka), a_tok,
                                                                        static_cast<const __nv_bfloat16 *>(kb), same ? 0 : b_tok,
