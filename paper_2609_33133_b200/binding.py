@@ -269,6 +269,58 @@ def run_forward_backward(plan: Plan, t, out):
                      out["dq_p"], None, None, out["ws"])
 
 
+class HostStep:
+    """The whole hot path for callers whose tensors live in (pinned) host memory: every input is copied to the device
+    and every result back, with the copies overlapped with the kernels as far as the data flow allows.  Three streams:
+    one for the host->device copies in the order the calls need them (prompt inputs, response inputs, dO_R, dO_P), the
+    caller's current stream for the four entry points (each waits only for its own inputs), one for the device->host
+    copies (each result leaves as soon as its call has finished).  The caller's stream has joined both copy streams
+    when `run` returns (asynchronously, like the entry points).  Copies and waits only: no arithmetic here."""
+
+    IN_ORDER = (("q_p", "k_p", "v_p"), ("q_r", "k_r", "v_r"), ("do_r",), ("do_p",))
+    OUT_ORDER = (("o_p", "lse_p"), ("o_r", "lse_r"), ("dq_r", "dk_r", "dv_r"), ("dq_p", "dk_p", "dv_p"))
+
+    def __init__(self, plan: Plan, dev_in, dev_out):
+        self.plan, self.t, self.out = plan, dev_in, dev_out
+        self.s_in, self.s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        self.ev_in = [torch.cuda.Event() for _ in self.IN_ORDER]
+        self.ev_done = [torch.cuda.Event() for _ in self.OUT_ORDER]
+        self.ev_start, self.ev_in_end, self.ev_out_end = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
+
+    def run(self, host_in, host_out):
+        plan, t, out = self.plan, self.t, self.out
+        main = torch.cuda.current_stream()
+        self.ev_start.record(main)                      # the device buffers are free once earlier work on `main` is done
+        self.s_in.wait_event(self.ev_start)
+        self.s_out.wait_event(self.ev_start)
+        with torch.cuda.stream(self.s_in):
+            for names, ev in zip(self.IN_ORDER, self.ev_in):
+                for k in names:
+                    t[k].copy_(host_in[k], non_blocking=True)
+                ev.record(self.s_in)
+            self.ev_in_end.record(self.s_in)
+        calls = (
+            lambda: plan.prefill_fwd(t["q_p"], t["k_p"], t["v_p"], out["o_p"], out["lse_p"], out["ws"]),
+            lambda: plan.replay_fwd(t["q_r"], t["k_r"], t["v_r"], t["k_p"], t["v_p"], out["o_r"], out["lse_r"], out["ws"]),
+            lambda: plan.replay_bwd(t["q_r"], t["k_r"], t["v_r"], t["k_p"], t["v_p"], out["o_r"], out["lse_r"], t["do_r"],
+                                    out["dq_r"], out["dk_r"], out["dv_r"], out["dk_p"], out["dv_p"], out["ws"]),
+            lambda: plan.prefill_bwd(t["q_p"], t["k_p"], t["v_p"], out["o_p"], out["lse_p"], t["do_p"], out["dk_p"], out["dv_p"],
+                                     out["dq_p"], None, None, out["ws"]),
+        )
+        for i, call in enumerate(calls):
+            main.wait_event(self.ev_in[i])
+            call()
+            self.ev_done[i].record(main)
+        with torch.cuda.stream(self.s_out):
+            for names, ev in zip(self.OUT_ORDER, self.ev_done):
+                self.s_out.wait_event(ev)
+                for k in names:
+                    host_out[k].copy_(out[k], non_blocking=True)
+            self.ev_out_end.record(self.s_out)
+        main.wait_event(self.ev_in_end)
+        main.wait_event(self.ev_out_end)
+
+
 def capture_step(plan: Plan, t, out):
     """The whole hot path captured once into a CUDA graph (the library allocates nothing and does not synchronise
     in its launch path); `graph.replay()` then re-runs it on the same buffers.  Pays off for launch-bound sizes."""

@@ -154,6 +154,24 @@ def test_flattened_baseline_matches_tree(B):
     pu.assert_parity({"dk_p": dk, "dv_p": dv, "dq_p": dq}, {k: ref[k] for k in ("dk_p", "dv_p", "dq_p")})
 
 
+def test_host_step_with_overlapped_copies_is_bitwise_the_plain_step(B):
+    """binding.HostStep (host tensors in, host tensors out, copies on their own streams) against the plain sequence."""
+    w = _wl("hoststep", [700, 130], [[300, 150, 420], [257]], 4, 2, 128, 72)
+    t_cpu = wl.make_tensors(w)
+    plain, plan = pu.run_gpu(B, w, t_cpu, flags=B.FLAG_ZERO_PROMPT_GRAD)
+    dev_in = {k: torch.zeros_like(v, device="cuda") for k, v in t_cpu.items()}
+    out = B.alloc_outputs(plan)
+    host_in = {k: v.pin_memory() for k, v in t_cpu.items()}
+    host_out = {k: torch.full(v.shape, float("nan"), dtype=v.dtype).pin_memory() for k, v in out.items() if k != "ws"}
+    step = B.HostStep(plan, dev_in, out)
+    for _ in range(3):                                   # back-to-back steps reuse the device buffers
+        step.run(host_in, host_out)
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0)
+    for k, v in host_out.items():
+        assert np.array_equal(v.float().numpy().astype(np.float64), plain[k]), k
+
+
 def test_cuda_graph_replay_is_bitwise_the_eager_step(B):
     """The four entry points capture into a CUDA graph (no allocation or synchronisation in the launch path)."""
     w = _wl("graph", [256], [[128] * 4], 4, 4, 64, 61)
