@@ -290,7 +290,8 @@ int augtree_last_device_status(const augtree_plan_t *plan, int *status, int *det
  *   plan's prompt keys over all given queries (complete for this shard: Eq. 2's sum is local to the shard's owner);
  *   dq_part [sumR,H_q,d] fp32 = this shard's contribution to dQ (written, not added); with include_own != 0 also
  *   the own-response part: dk_r, dv_r (bf16) written and the causal range included in dq_part; with
- *   include_own == 0, dk_r and dv_r may be NULL and k_r, v_r are not read.
+ *   include_own == 0, dk_r and dv_r may be NULL, and k_r, v_r are not read (they must still be valid device
+ *   pointers of the plan's response shape: a tensor map is encoded over them).
  */
 int augtree_replay_fwd_state(const augtree_plan_t *plan, const void *q_r, const void *k_r, const void *v_r,
                              const void *k_p, const void *v_p, float *state_o, float *state_lse, int include_own,
