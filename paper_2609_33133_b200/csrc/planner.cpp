@@ -9,6 +9,7 @@
 #include <cmath>
 #include <cstdint>
 #include <limits>
+#include <map>
 #include <numeric>
 #include <vector>
 
@@ -73,9 +74,10 @@ struct ExactGrid {
     return round_best[b][full] < kInf;
   }
 
-  void unpack(int32_t *round_out, int32_t *lane_out) const {
+  // placement that attains round_best[rounds][all units] (rounds <= b)
+  void unpack(int32_t *round_out, int32_t *lane_out, int rounds = -1) const {
     uint32_t S = (1u << U) - 1;
-    int t = b, round = 0;
+    int t = rounds < 0 ? b : rounds, round = 0;
     while (S) {
       const uint32_t R = round_pick[t][S];
       uint32_t L = R;
@@ -215,6 +217,7 @@ static int plan_tree_impl(const augtree_tree_t *t, const augtree_profile_t *pr, 
   augtree_choice_t best = {};
   std::vector<int32_t> rounds(G), lanes(G), best_rounds(G), best_lanes(G);
   int n_cand = 0;
+  std::map<std::pair<int, int64_t>, ExactGrid> dp_cache;
   for (int di = 0; di < t->n_degrees; ++di) {
     const int d = t->degrees[di];
     if (d < 1 || d > 65536) return AUGTREE_ERR_INVALID_ARG;
@@ -251,13 +254,36 @@ static int plan_tree_impl(const augtree_tree_t *t, const augtree_profile_t *pr, 
           cap = (int64_t)std::floor(room / pr->mem_resp);
           if (cap < 1) { n_cand += (int)std::min<int64_t>(b_max, cdiv64(G, s)); continue; }   // not even one token fits
         }
-        for (int b = 1; b <= std::min<int64_t>(b_max, cdiv64(G, s)); ++b) {
+        // Up to the exact solver's limit one dynamic program per (primitive, s) serves every round count: its table
+        // round_best[b][all units] is the optimum of Eq. 6 with at most b rounds.  Above the limit the greedy runs per b.
+        const int b_hi = (int)std::min<int64_t>(b_max, cdiv64(G, s));
+        const int exact_cap = std::min(t->exact_max_units > 0 ? t->exact_max_units : 12, kHardMaxExact);
+        const bool use_dp = G <= exact_cap;
+        // the program depends on (s, cell limit) alone: shared by degrees and primitives that agree on both
+        ExactGrid *dp_ptr = nullptr;
+        if (use_dp) {
+          auto key = std::make_pair(s, cap);
+          auto it = dp_cache.find(key);
+          if (it == dp_cache.end()) {
+            it = dp_cache.emplace(key, ExactGrid()).first;
+            it->second.U = G; it->second.b = (int)std::min<int64_t>(b_max, G); it->second.s = std::min(s, G);
+            it->second.solve(w.data(), m.data(), cap);
+          }
+          dp_ptr = &it->second;
+        }
+        for (int b = 1; b <= b_hi; ++b) {
           ++n_cand;
           int64_t work = 0;
           int32_t exact = 0;
-          const int r = assign_grid_impl(w.data(), m.data(), G, b, s, cap, t->exact_max_units, rounds.data(), lanes.data(), &work, &exact);
-          if (r == AUGTREE_ERR_UNSUPPORTED) continue;  // the units do not fit this grid
-          if (r) return r;
+          if (use_dp) {
+            work = dp_ptr->round_best[b][(1u << G) - 1];
+            if (work >= kInf) continue;  // the units do not fit this grid
+            exact = 1;
+          } else {
+            const int r = assign_grid_impl(w.data(), m.data(), G, b, s, cap, t->exact_max_units, rounds.data(), lanes.data(), &work, &exact);
+            if (r == AUGTREE_ERR_UNSUPPORTED) continue;
+            if (r) return r;
+          }
           const double L = (double)(cdiv64(G, (int64_t)b * s) * r_max);
           double replay, gamma;
           int d_eff;
@@ -278,6 +304,7 @@ static int plan_tree_impl(const augtree_tree_t *t, const augtree_profile_t *pr, 
           if (!have || cost < best.cost) {
             have = true;
             best.cost = cost; best.degree = d; best.primitive = primitive; best.rounds = b; best.lanes = s; best.solved_exactly = exact;
+            if (use_dp) dp_ptr->unpack(rounds.data(), lanes.data(), b);
             best_rounds = rounds; best_lanes = lanes;
           }
         }
