@@ -82,43 +82,51 @@ def _branch_len_by_group(w, lay: RankLayout, branches):
 
 
 class CudaBackend:
-    """The per-rank compute steps as library calls (one plan per (rank, branch set); plans are cached)."""
+    """The per-rank compute steps as library calls.  A call is described by the lengths of the key shards it holds (one
+    per group) and of the response branches it is given (per group); plans are cached by that description."""
 
     def __init__(self, binding, w, device=0):
         self.B, self.w, self.device, self._plans = binding, w, device, {}
 
-    def _plan(self, lay, branches):
-        key = (lay.rank, tuple(branches))
+    def _plan(self, shard_len, branch_lens):
+        key = (tuple(shard_len), tuple(tuple(b) for b in branch_lens))
         if key not in self._plans:
             w = self.w
-            self._plans[key] = self.B.Plan(lay.shard_len, _branch_len_by_group(w, lay, branches), w.h_q, w.h_kv, w.head_dim,
-                                           device=self.device)
+            self._plans[key] = self.B.Plan(list(shard_len), [list(b) for b in branch_lens], w.h_q, w.h_kv, w.head_dim, device=self.device)
         return self._plans[key]
 
     def _ws(self, plan):
         return torch.empty(max(plan.ws_fwd_bytes, plan.ws_bwd_bytes, 256), device="cuda", dtype=torch.uint8)
 
-    def fwd_state(self, lay, branches, include_own, q, k_r, v_r, k_p, v_p):
-        plan = self._plan(lay, branches)
+    def fwd_state_on(self, shard_len, branch_lens, include_own, q, k_r, v_r, k_p, v_p):
+        plan = self._plan(shard_len, branch_lens)
         so = torch.empty((plan.total_r, self.w.h_q, self.w.head_dim), device="cuda", dtype=torch.float32)
         sl = torch.empty((self.w.h_q, plan.total_r), device="cuda", dtype=torch.float32)
         plan.replay_fwd_state(q, k_r, v_r, k_p, v_p, so, sl, include_own, self._ws(plan))
         return so, sl
 
-    def merge(self, full_plan, states_o, states_lse):
-        o = torch.empty((full_plan.total_r, self.w.h_q, self.w.head_dim), device="cuda", dtype=torch.bfloat16)
-        lse = torch.empty((self.w.h_q, full_plan.total_r), device="cuda", dtype=torch.float32)
-        full_plan.merge_states(states_o, states_lse, o, lse)
+    def merge(self, _unused, states_o, states_lse):
+        n = states_o[0].shape[0]
+        plan = self._plan([1], [[n]])                     # the merge only needs the row count and the head geometry
+        o = torch.empty((n, self.w.h_q, self.w.head_dim), device="cuda", dtype=torch.bfloat16)
+        lse = torch.empty((self.w.h_q, n), device="cuda", dtype=torch.float32)
+        plan.merge_states(states_o, states_lse, o, lse)
         return o, lse
 
-    def bwd_state(self, lay, branches, include_own, q, k_r, v_r, k_p, v_p, o, lse, do, dkp, dvp):
-        plan = self._plan(lay, branches)
+    def bwd_state_on(self, shard_len, branch_lens, include_own, q, k_r, v_r, k_p, v_p, o, lse, do, dkp, dvp):
+        plan = self._plan(shard_len, branch_lens)
         hq, hkv, d = self.w.h_q, self.w.h_kv, self.w.head_dim
         dq = torch.empty((plan.total_r, hq, d), device="cuda", dtype=torch.float32)
         dk = torch.empty((plan.total_r, hkv, d), device="cuda", dtype=torch.bfloat16)
         dv = torch.empty_like(dk)
         plan.replay_bwd_state(q, k_r, v_r, k_p, v_p, o, lse, do, dq, dk, dv, dkp, dvp, include_own, self._ws(plan))
         return dq, dk, dv
+
+    def fwd_state(self, lay, branches, include_own, *tensors):
+        return self.fwd_state_on(lay.shard_len, _branch_len_by_group(self.w, lay, branches), include_own, *tensors)
+
+    def bwd_state(self, lay, branches, include_own, *tensors):
+        return self.bwd_state_on(lay.shard_len, _branch_len_by_group(self.w, lay, branches), include_own, *tensors)
 
     def status_ok(self):
         return all(p.device_status() == (0, 0) for p in self._plans.values())
@@ -166,13 +174,12 @@ def moveq_emulate(binding, w, t, world: int, device=0):
     exchange that follows it).  `t`: the workload's full tensors on the device.  Returns o_r, lse_r, dq_r, dk_r, dv_r
     and the prompt-KV gradient seeds dk_p, dv_p (fp32, replay part only: the prefill backward adds its own)."""
     backend = CudaBackend(binding, w, device)
-    full_plan = binding.Plan(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, device=device)
     lays = [make_layout(w, r, world) for r in range(world)]
     shard = [(t["k_p"][torch.as_tensor(l.prompt_idx, device="cuda")].contiguous(),
               t["v_p"][torch.as_tensor(l.prompt_idx, device="cuda")].contiguous()) for l in lays]
     # forward: queries known everywhere (the exchange: all-gather of the owners' query rows) -> states -> merge on the owners
     states = [fwd_compute(backend, w, lays[r], t["q_r"], t["k_r"], t["v_r"], *shard[r]) for r in range(world)]
-    o, lse = backend.merge(full_plan, [s[0] for s in states], [s[1] for s in states])
+    o, lse = backend.merge(None, [s[0] for s in states], [s[1] for s in states])
     # backward: merged O, LSE and dO known everywhere -> per-rank gradients -> dQ summed back to the owners
     parts = [bwd_compute(backend, w, lays[r], t["q_r"], t["k_r"], t["v_r"], *shard[r], o, lse, t["do_r"]) for r in range(world)]
     dq = torch.stack([p[0] for p in parts]).sum(dim=0)            # the reverse exchange: sum over KV owners, fixed rank order
@@ -185,7 +192,7 @@ def moveq_emulate(binding, w, t, world: int, device=0):
         dk_p[idx] = parts[r][3]
         dv_p[idx] = parts[r][4]
     torch.cuda.synchronize()
-    if not backend.status_ok() or full_plan.device_status() != (0, 0):
+    if not backend.status_ok():
         raise RuntimeError("device status")
     return {"o_r": o, "lse_r": lse, "dq_r": dq, "dk_r": dk_r, "dv_r": dv_r, "dk_p": dk_p, "dv_p": dv_p}
 
@@ -298,3 +305,55 @@ def treemovekv_emulate(binding, w, t, s: int, d_lane: int, rounds: int = 1, devi
         raise RuntimeError("device status")
     out["placement"] = (x_round, x_lane)
     return out
+
+
+def _ring_pass(dist, rank, world, tensors):
+    """One ring step: every tensor of `tensors` goes to rank + 1 and is replaced by what rank - 1 sends.  Shapes may differ
+    from rank to rank (shards differ by a token), so the sizes are exchanged with the data: first dimension only."""
+    nxt, prv = (rank + 1) % world, (rank - 1) % world
+    n_out = torch.tensor([t.shape[0] for t in tensors], dtype=torch.int64)
+    n_in = torch.empty_like(n_out)
+    for req in dist.batch_isend_irecv([dist.P2POp(dist.isend, n_out, nxt), dist.P2POp(dist.irecv, n_in, prv)]):
+        req.wait()
+    recv = [torch.empty((int(n),) + tuple(t.shape[1:]), dtype=t.dtype, device=t.device) for n, t in zip(n_in.tolist(), tensors)]
+    ops = [dist.P2POp(dist.isend, t.contiguous(), nxt) for t in tensors] + [dist.P2POp(dist.irecv, r, prv) for r in recv]
+    for req in dist.batch_isend_irecv(ops):
+        req.wait()
+    return recv
+
+
+def treemovekv_rank(dist, backend, w, rank: int, world: int, local: Dict[str, torch.Tensor]):
+    """One rank of a multi-process TreeMoveKV lane (the whole process group is one lane, one round, one replay tree).
+    `local`: k_p, v_p = this rank's prompt-KV shard; q_r, k_r, v_r, do_r = the rows of the branches it owns (branch k
+    belongs to rank k % world), packed in branch order.  The prompt-KV shards go round the ring twice: once for the
+    forward states, once more with their fp32 gradient accumulators, which are home again after the last step.
+    Returns o_r, lse_r, dq_r, dk_r, dv_r for the owned rows and dk_p, dv_p of the rank's own shard."""
+    if w.n_groups != 1:
+        raise ValueError("one replay tree at a time")
+    mine = [[r for k, r in enumerate(w.branch_len[0]) if k % world == rank]]
+    q, k_r, v_r, do = local["q_r"], local["k_r"], local["v_r"], local["do_r"]
+    have = bool(mine[0])
+    kp, vp = local["k_p"], local["v_p"]
+    states_o, states_l = [], []
+    for stage in range(world):                              # forward ring
+        if have:
+            so, sl = backend.fwd_state_on([kp.shape[0]], mine, stage == 0, q, k_r, v_r, kp, vp)
+            states_o.append(so); states_l.append(sl)
+        kp, vp = _ring_pass(dist, rank, world, [kp, vp])   # after `world` passes the own shard is back
+    res = {}
+    if have:
+        o, lse = backend.merge(None, states_o, states_l)
+        dq = torch.zeros(q.shape, dtype=torch.float32, device=q.device)
+    gk = torch.zeros(kp.shape, dtype=torch.float32, device=kp.device)
+    gv = torch.zeros_like(gk)
+    for stage in range(world):                              # backward ring: shards travel with their accumulators
+        if have:
+            part, dk, dv = backend.bwd_state_on([kp.shape[0]], mine, stage == 0, q, k_r, v_r, kp, vp, o, lse, do, gk, gv)
+            dq += part
+            if stage == 0:
+                res.update(dk_r=dk, dv_r=dv)
+        kp, vp, gk, gv = _ring_pass(dist, rank, world, [kp, vp, gk, gv])
+    if have:
+        res.update(o_r=o, lse_r=lse, dq_r=dq)
+    res.update(dk_p=gk, dv_p=gv)
+    return res

@@ -25,21 +25,27 @@ class OracleBackend:
     def __init__(self, w):
         self.w, self.scale, self.rep = w, 1.0 / np.sqrt(w.head_dim), w.h_q // w.h_kv
 
-    def _walk(self, lay, branches):
-        """(rows of the call's packed query tensor, group index, offset of the group's shard in the rank's prompt tensor)."""
-        off_p = np.concatenate([[0], np.cumsum(lay.shard_len)])
+    @staticmethod
+    def _walk(shard_len, branch_lens):
+        """(rows of the call's packed query tensor, rows of the call's key-shard tensor) branch by branch, group-major."""
+        off_p = np.concatenate([[0], np.cumsum(shard_len)])
         pos = 0
-        for i in branches:
-            n = len(lay.branch_tok[i])
-            g = lay.branch_group[i]
-            yield slice(pos, pos + n), slice(int(off_p[g]), int(off_p[g + 1]))
-            pos += n
+        for g, lens in enumerate(branch_lens):
+            for n in lens:
+                yield slice(pos, pos + n), slice(int(off_p[g]), int(off_p[g + 1]))
+                pos += n
 
-    def fwd_state(self, lay, branches, include_own, q, k_r, v_r, k_p, v_p):
+    def fwd_state(self, lay, branches, include_own, *tensors):
+        return self.fwd_state_on(lay.shard_len, cp._branch_len_by_group(self.w, lay, branches), include_own, *tensors)
+
+    def bwd_state(self, lay, branches, include_own, *tensors):
+        return self.bwd_state_on(lay.shard_len, cp._branch_len_by_group(self.w, lay, branches), include_own, *tensors)
+
+    def fwd_state_on(self, shard_len, branch_lens, include_own, q, k_r, v_r, k_p, v_p):
         f = lambda x: x.double().numpy()
         q, k_r, v_r, k_p, v_p = f(q), f(k_r), f(v_r), f(k_p), f(v_p)
         so = np.zeros((q.shape[0], self.w.h_q, self.w.head_dim)); sl = np.zeros((self.w.h_q, q.shape[0]))
-        for rows, shard in self._walk(lay, branches):
+        for rows, shard in self._walk(shard_len, branch_lens):
             n = rows.stop - rows.start
             for h in range(self.w.h_q):
                 c = h // self.rep
@@ -61,12 +67,12 @@ class OracleBackend:
         o = np.stack([x[0] for x in fin], axis=1); lse = np.stack([x[1] for x in fin], axis=0)
         return torch.from_numpy(o).to(torch.bfloat16), torch.from_numpy(lse).float()
 
-    def bwd_state(self, lay, branches, include_own, q, k_r, v_r, k_p, v_p, o, lse, do, dkp, dvp):
+    def bwd_state_on(self, shard_len, branch_lens, include_own, q, k_r, v_r, k_p, v_p, o, lse, do, dkp, dvp):
         f = lambda x: x.double().numpy()
         q, k_r, v_r, k_p, v_p, o, lse, do = f(q), f(k_r), f(v_r), f(k_p), f(v_p), f(o), f(lse), f(do)
         dq = np.zeros_like(q); dk = np.zeros_like(k_r); dv = np.zeros_like(v_r)
         gk = np.zeros_like(k_p); gv = np.zeros_like(v_p)
-        for rows, shard in self._walk(lay, branches):
+        for rows, shard in self._walk(shard_len, branch_lens):
             n = rows.stop - rows.start
             for h in range(self.w.h_q):
                 c = h // self.rep
@@ -135,3 +141,53 @@ def test_moveq_exchange_on_two_gloo_ranks():
         assert np.abs(out["dk_p"] - ref["dk_p"][idx]).max() <= 1e-2 and np.abs(out["dv_p"] - ref["dv_p"][idx]).max() <= 1e-2
     covered = np.sort(np.concatenate([r[2] for r in res]))
     assert np.array_equal(covered, np.arange(W.total_prompt))
+
+
+W_RING = wl.Workload("tmkv-gloo", [41], [[9, 20, 5, 16, 7]], 4, 2, 16, 6)
+
+
+def _ring_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    w = W_RING
+    t = wl.make_tensors(w)
+    cu = np.concatenate([[0], np.cumsum(w.branch_len[0])])
+    rows = [np.arange(cu[k], cu[k + 1]) for k in range(len(w.branch_len[0])) if k % world == rank]
+    rows = torch.as_tensor(np.concatenate(rows)) if rows else torch.zeros(0, dtype=torch.int64)
+    a, b = cp.shard_bounds(w.prompt_len[0], world)[rank]
+    local = {k: t[k][rows].contiguous() for k in ("q_r", "k_r", "v_r", "do_r")}
+    local.update(k_p=t["k_p"][a:b].contiguous(), v_p=t["v_p"][a:b].contiguous())
+    res = cp.treemovekv_rank(dist, OracleBackend(w), w, rank, world, local)
+    out.put((rank, {k: v.float().numpy() for k, v in res.items()}, rows.numpy(), (a, b)))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_treemovekv_ring_on_three_gloo_ranks():
+    """The lane-local KV ring of TreeMoveKV: prompt-KV shards passed from rank to rank (P2P send / receive), the states of
+    a rank's own queries merged after the last stage, the shards' gradient accumulators home after a second round."""
+    world, port = 3, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_ring_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted((q.get(timeout=180) for _ in range(world)), key=lambda x: x[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    w = W_RING
+    t = wl.make_tensors(w)
+    tb = ora.TreeBatch(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim)
+    f = lambda x: x.float().numpy().astype(np.float64)
+    ref = ora.tree_attention_fwd_bwd(tb, f(t["q_p"]), f(t["k_p"]), f(t["v_p"]), np.zeros_like(f(t["do_p"])), f(t["q_r"]), f(t["k_r"]),
+                                     f(t["v_r"]), f(t["do_r"]))
+    seen = []
+    for rank, out, rows, (a, b) in res:
+        seen += rows.tolist()
+        for k, tol in (("o_r", 2e-2), ("dq_r", 1e-2), ("dk_r", 5e-2), ("dv_r", 5e-2)):
+            assert np.abs(out[k] - ref[k][rows]).max() <= tol, (rank, k)
+        assert np.abs(out["lse_r"] - ref["lse_r"][:, rows]).max() <= 1e-5
+        # the accumulators that came home are those of the rank's own shard, summed over every rank's queries (Eq. 2)
+        assert np.abs(out["dk_p"] - ref["dk_p"][a:b]).max() <= 1e-2 and np.abs(out["dv_p"] - ref["dv_p"][a:b]).max() <= 1e-2
+    assert sorted(seen) == list(range(w.total_response))
