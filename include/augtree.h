@@ -275,7 +275,10 @@ int augtree_last_device_status(const augtree_plan_t *plan, int *status, int *det
  * owns the query; in the backward pass every shard owner computes its shard's dK, dV and its contribution to dQ
  * from the merged LSE, and the dQ contributions are summed on the way back ("its custom autograd operator applies
  * the reverse communication", Sec. 3.3).  These three calls are the per-rank compute steps; moving queries,
- * states and gradients between ranks is the caller's (NCCL or peer copies, no multicast loads).
+ * states and gradients between ranks is the caller's (NCCL or peer copies, no multicast loads).  state_o,
+ * state_lse and dq_part are written with plain global stores from the tile kernels' epilogues, so they may be
+ * peer-mapped memory of the rank that will merge them: the exchange then happens as the tiles finish.  Inputs
+ * are read through TMA and must be this device's own memory.
  *
  * The plan describes THIS RANK'S view: its "prompt" is the shard of unmasked keys it holds (k_p, v_p: a prompt-KV
  * shard, or any keys every given query may see in full), its branches are the response queries it is given.
