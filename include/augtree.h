@@ -152,6 +152,18 @@ int augtree_plan_destroy(augtree_plan_t *plan);
 int augtree_plan_workspace_bytes(const augtree_plan_t *plan, size_t *fwd_bytes, size_t *bwd_bytes);
 
 /*
+ * Backward scratch size from which the backward calls take the hand-off path.  The textbook backward of
+ * attention is five GEMMs per (query tile, KV tile) pair; with bwd_bytes of scratch the two kernels of a
+ * backward call (key side: dK, dV; query side: dQ) each recompute S and dP, seven GEMMs in all.  A call
+ * given ws_bytes >= *bytes instead has the key-side kernel store dS (bf16, 32 KB per pair and query head:
+ * *bytes = bwd_bytes + that, the larger of the two backward calls) and the query-side kernel compute
+ * dQ = sum dS K from it: five GEMMs, at the price of writing and reading the scratch once.  Both paths give
+ * dK, dV bit for bit the same and dQ from the same bf16 dS values summed in the same order.  *bytes is
+ * SIZE_MAX for a plan too large to index; the choice is the caller's, per call, through ws_bytes.
+ */
+int augtree_plan_bwd_handoff_bytes(const augtree_plan_t *plan, size_t *bytes);
+
+/*
  * Copy one metadata table to host memory.  With host_dst == NULL only *bytes
  * is set.  Otherwise *bytes is the capacity on entry and the size on return.
  * Item layouts (int32 each):

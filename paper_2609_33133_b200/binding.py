@@ -34,7 +34,7 @@ EXPORTS = ["augtree_plan_create", "augtree_plan_destroy", "augtree_plan_workspac
            "augtree_last_device_status", "augtree_launch_count", "augtree_status_string",
            "augtree_set_timing", "augtree_get_kernel_time", "augtree_replay_fwd_static", "augtree_assign_grid",
            "augtree_items_completed", "augtree_plan_tree", "augtree_replay_fwd_state", "augtree_merge_states",
-           "augtree_replay_bwd_state"]
+           "augtree_replay_bwd_state", "augtree_plan_bwd_handoff_bytes"]
 
 
 class Desc(C.Structure):
@@ -50,6 +50,7 @@ _i64p, _i32p = C.POINTER(C.c_int64), C.POINTER(C.c_int32)
 lib.augtree_plan_create.argtypes = [C.POINTER(Desc), C.c_int, C.POINTER(_vp)]
 lib.augtree_plan_destroy.argtypes = [_vp]
 lib.augtree_plan_workspace_bytes.argtypes = [_vp, C.POINTER(_sz), C.POINTER(_sz)]
+lib.augtree_plan_bwd_handoff_bytes.argtypes = [_vp, C.POINTER(_sz)]
 lib.augtree_plan_metadata.argtypes = [_vp, C.c_int, _vp, C.POINTER(_sz)]
 lib.augtree_prefill_fwd.argtypes = [_vp] + [_vp] * 5 + [_vp, _sz, _vp]
 lib.augtree_replay_fwd.argtypes = [_vp] + [_vp] * 7 + [_vp, _sz, _vp]
@@ -141,6 +142,9 @@ def launch_count() -> int:
     return int(lib.augtree_launch_count())
 
 
+HANDOFF_LIMIT_BYTES = 0   # default ceiling on the backward hand-off scratch: 0 = recomputing path
+
+
 class Plan:
     """Owns an augtree_plan_t.  device=None builds a host-only plan (metadata queries only)."""
 
@@ -164,6 +168,14 @@ class Plan:
         f, b = _sz(), _sz()
         _check(lib.augtree_plan_workspace_bytes(self._h, C.byref(f), C.byref(b)), "workspace_bytes")
         self.ws_fwd_bytes, self.ws_bwd_bytes = f.value, b.value
+        _check(lib.augtree_plan_bwd_handoff_bytes(self._h, C.byref(b)), "bwd_handoff_bytes")
+        self.ws_bwd_handoff_bytes = b.value
+
+    def workspace_bytes(self, handoff_limit=HANDOFF_LIMIT_BYTES) -> int:
+        """Scratch for all four calls.  The backward calls take the dS hand-off path (five GEMMs per tile pair instead
+        of seven) when its scratch fits under `handoff_limit` bytes, else the recomputing path."""
+        need = max(self.ws_fwd_bytes, self.ws_bwd_bytes, 256)
+        return max(need, self.ws_bwd_handoff_bytes) if self.ws_bwd_handoff_bytes <= handoff_limit else need
 
     def __del__(self):
         h = getattr(self, "_h", None)
@@ -245,7 +257,7 @@ class Plan:
         return s.value, d.value
 
 
-def alloc_outputs(plan: Plan, device="cuda"):
+def alloc_outputs(plan: Plan, device="cuda", handoff_limit=HANDOFF_LIMIT_BYTES):
     """Device buffers for one forward + backward pass (allocation only)."""
     hq, hkv, d = plan.h_q, plan.h_kv, plan.head_dim
     bf, f32 = torch.bfloat16, torch.float32
@@ -255,7 +267,7 @@ def alloc_outputs(plan: Plan, device="cuda"):
         "o_p": e(tp, hq, d), "lse_p": e(hq, tp, dt=f32), "o_r": e(tr, hq, d), "lse_r": e(hq, tr, dt=f32),
         "dq_p": e(tp, hq, d), "dq_r": e(tr, hq, d), "dk_r": e(tr, hkv, d), "dv_r": e(tr, hkv, d),
         "dk_p": torch.zeros((tp, hkv, d), device=device, dtype=f32), "dv_p": torch.zeros((tp, hkv, d), device=device, dtype=f32),
-        "ws": torch.empty(max(plan.ws_fwd_bytes, plan.ws_bwd_bytes, 256), device=device, dtype=torch.uint8),
+        "ws": torch.empty(plan.workspace_bytes(handoff_limit), device=device, dtype=torch.uint8),
     }
 
 

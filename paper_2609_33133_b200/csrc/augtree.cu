@@ -10,6 +10,7 @@
 
 #include "bwd_kernel.cuh"
 #include "dq_kernel.cuh"
+#include "dql_kernel.cuh"
 #include "fwd_kernel.cuh"
 #include "plan.h"
 
@@ -54,6 +55,22 @@ int make_map(CUtensorMap *m, const void *ptr, long long tokens, int heads, int d
   const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)heads, (cuuint64_t)tokens};
   const cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)heads * d * 2};
   const cuuint32_t box[3] = {64, 1, 128};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? AUGTREE_OK : AUGTREE_ERR_CUDA;
+}
+
+// Tensor map over the dS hand-off scratch: [slots][128 keys][128 queries] bf16, one box = 64 queries of all 128
+// keys of one slot (the MN-major A operand of the query-side GEMM, 128-byte swizzle).
+int make_ds_map(CUtensorMap *m, const void *ptr, long long slots) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return AUGTREE_ERR_CUDA;
+  if (slots < 1) slots = 1;
+  const cuuint64_t dims[3] = {128, 128, (cuuint64_t)slots};
+  const cuuint64_t strides[2] = {256, 32768};
+  const cuuint32_t box[3] = {64, 128, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -158,13 +175,19 @@ struct BwdArgs {
   const void *ka, *va; long long a_tok;
   int no_own = 0;           // partial-state variant: only the plan's prompt keys (mode-1 items, no causal range in dQ)
   float *dq_f32 = nullptr;  // partial-state variant: fp32 dQ contribution
+  const int32_t *d_pairs = nullptr;  // dS hand-off table of the call's query tiles
+  long long ds_slots = 0;            // (KV tile, query tile) pairs per head of the call
 };
 
 // One backward call: row statistics, then the key-side kernel (dK, dV), then the query-side kernel (dQ).
+// With scratch for it (ws_bytes >= the plan's hand-off size) the key-side kernel also stores dS and the
+// query side is one GEMM per pair (dql_kernel); otherwise the query side recomputes S and dP (dq_kernel).
 template <int D>
-int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *ws, cudaStream_t st) {
+int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *ws, size_t ws_bytes, cudaStream_t st) {
   if (a.q_tok == 0) return AUGTREE_OK;
   float *stats = static_cast<float *>(ws);
+  const bool handoff = ws_bytes >= pl->ws_bwd_handoff && s.n_items() > 0 && a.dq_sched->n_items() > 0;
+  __nv_bfloat16 *ds = handoff ? reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(ws) + pl->ws_bwd) : nullptr;
   {
     const dim3 grid((unsigned)a.n_tiles, (unsigned)pl->h_q);
     bwd_preprocess_kernel<D><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(a.o), static_cast<const __nv_bfloat16 *>(a.d_o),
@@ -190,6 +213,7 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     p.wait_budget = wait_budget(pl); p.kind = kind;
     p.test_flags = (pl->flags & AUGTREE_FLAG_TEST_SKIP_BWD_LOAD) ? TEST_SKIP_BWD_LOAD : 0;
     p.no_own = a.no_own;
+    p.ds_out = ds; p.pair_tab = reinterpret_cast<const int4 *>(a.d_pairs);
     long long n_run = s.n_items();
     if (a.no_own) {
       n_run = 0;
@@ -202,7 +226,22 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return AUGTREE_ERR_CUDA;
   }
-  if (a.dq_sched->n_items() > 0) {
+  if (handoff) {
+    CUtensorMap mds, mka;
+    if ((r = make_ds_map(&mds, ds, a.ds_slots * pl->h_q))) return r;
+    if ((r = make_map(&mka, a.ka, a.a_tok, pl->h_kv, D))) return r;
+    DqlParams p;
+    p.items = a.dq_sched->d_items; p.lane_ptr = a.dq_sched->d_lane_ptr; p.pair_tab = reinterpret_cast<const int4 *>(a.d_pairs);
+    p.dq = static_cast<__nv_bfloat16 *>(a.dq); p.dq_f32 = a.dq_f32; p.h_q = pl->h_q; p.no_own = a.no_own;
+    p.status = pl->d_status;
+    const int kind = (int)(a.dq_sched - pl->sched);
+    p.wait_budget = wait_budget(pl); p.kind = kind;
+    pl->launched_items[kind] += a.dq_sched->n_items();
+    timing_mark(pl, kind, false, st);
+    dql_kernel<D><<<pl->n_lanes, kDqlThreads, DqlSmem<D>::kBytes, st>>>(mds, mka, mk0, p);
+    timing_mark(pl, kind, true, st);
+    ++g_launches;
+  } else if (a.dq_sched->n_items() > 0) {
     CUtensorMap mka, mva;
     if ((r = make_map(&mka, a.ka, a.a_tok, pl->h_kv, D))) return r;
     if ((r = make_map(&mva, a.va, a.a_tok, pl->h_kv, D))) return r;
@@ -257,7 +296,8 @@ template <int D>
 int set_kernel_attributes() {
   if (cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kBytes) != cudaSuccess ||
       cudaFuncSetAttribute(bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kBytes) != cudaSuccess ||
-      cudaFuncSetAttribute(dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<D>::kBytes) != cudaSuccess)
+      cudaFuncSetAttribute(dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<D>::kBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(dql_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqlSmem<D>::kBytes) != cudaSuccess)
     return AUGTREE_ERR_CUDA;
   return AUGTREE_OK;
 }
@@ -308,6 +348,8 @@ int augtree_plan_create(const augtree_desc_t *desc, int device, augtree_plan_t *
     if (!r) r = upload(pl->cu_r, &pl->d_cu_r);
     if (!r) r = upload(pl->tiles_replay, &pl->d_tiles_replay);
     if (!r) r = upload(pl->tiles_prefill, &pl->d_tiles_prefill);
+    if (!r) r = upload(pl->pairs_replay, &pl->d_pairs_replay);
+    if (!r) r = upload(pl->pairs_prefill, &pl->d_pairs_prefill);
     if (!r) {
       if (cudaMalloc(&pl->d_status, kStatusInts * sizeof(int)) != cudaSuccess ||
           cudaMemset(pl->d_status, 0, kStatusInts * sizeof(int)) != cudaSuccess)
@@ -329,6 +371,7 @@ int augtree_plan_destroy(augtree_plan_t *pl) {
     for (int k = 0; k < SCHED_COUNT; ++k) { cudaFree(pl->sched[k].d_items); cudaFree(pl->sched[k].d_lane_ptr); }
     cudaFree(pl->d_seg_replay); cudaFree(pl->d_seg_prefill); cudaFree(pl->d_branch_group); cudaFree(pl->d_group_splits);
     cudaFree(pl->d_cu_r); cudaFree(pl->d_status); cudaFree(pl->d_tiles_replay); cudaFree(pl->d_tiles_prefill);
+    cudaFree(pl->d_pairs_replay); cudaFree(pl->d_pairs_prefill);
     if (pl->timing) {
       for (int k = 0; k < SCHED_COUNT; ++k)
         for (void *e : pl->timing->ev[k]) cudaEventDestroy(static_cast<cudaEvent_t>(e));
@@ -344,6 +387,12 @@ int augtree_plan_workspace_bytes(const augtree_plan_t *pl, size_t *fwd, size_t *
   if (!pl) return AUGTREE_ERR_INVALID_ARG;
   if (fwd) *fwd = pl->ws_fwd;
   if (bwd) *bwd = pl->ws_bwd;
+  return AUGTREE_OK;
+}
+
+int augtree_plan_bwd_handoff_bytes(const augtree_plan_t *pl, size_t *bytes) {
+  if (!pl || !bytes) return AUGTREE_ERR_INVALID_ARG;
+  *bytes = pl->ws_bwd_handoff;
   return AUGTREE_OK;
 }
 
@@ -522,9 +571,10 @@ int augtree_replay_bwd_state(const augtree_plan_t *pl, const void *q_r, const vo
   a.dq = nullptr; a.dk_out = dk_r; a.dv_out = dv_r; a.dk_acc = dkp_acc; a.dv_acc = dvp_acc; a.causal_fp32 = 0;
   a.d_segs = pl->d_seg_replay; a.d_tiles = pl->d_tiles_replay; a.n_tiles = (long long)pl->tiles_replay.size() / 2;
   a.dq_sched = &pl->sched[SCHED_REPLAY_DQ]; a.ka = k_p; a.va = v_p; a.a_tok = pl->total_p;
+  a.d_pairs = pl->d_pairs_replay; a.ds_slots = pl->ds_slots_replay;
   a.no_own = include_own ? 0 : 1; a.dq_f32 = dq_part;
   const Sched &s = pl->sched[SCHED_REPLAY_BWD];
-  return pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, st) : launch_bwd<64>(pl, s, a, ws, st);
+  return pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, ws_bytes, st) : launch_bwd<64>(pl, s, a, ws, ws_bytes, st);
 }
 
 int augtree_replay_bwd(const augtree_plan_t *pl, const void *q_r, const void *k_r, const void *v_r, const void *k_p,
@@ -551,8 +601,9 @@ int augtree_replay_bwd(const augtree_plan_t *pl, const void *q_r, const void *k_
   a.dq = dq_r; a.dk_out = dk_r; a.dv_out = dv_r; a.dk_acc = dkp_acc; a.dv_acc = dvp_acc; a.causal_fp32 = 0;
   a.d_segs = pl->d_seg_replay; a.d_tiles = pl->d_tiles_replay; a.n_tiles = (long long)pl->tiles_replay.size() / 2;
   a.dq_sched = &pl->sched[SCHED_REPLAY_DQ]; a.ka = k_p; a.va = v_p; a.a_tok = pl->total_p;
+  a.d_pairs = pl->d_pairs_replay; a.ds_slots = pl->ds_slots_replay;
   const Sched &s = pl->sched[SCHED_REPLAY_BWD];
-  return pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, st) : launch_bwd<64>(pl, s, a, ws, st);
+  return pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, ws_bytes, st) : launch_bwd<64>(pl, s, a, ws, ws_bytes, st);
 }
 
 int augtree_prefill_bwd(const augtree_plan_t *pl, const void *q_p, const void *k_p, const void *v_p, const void *o_p,
@@ -572,8 +623,9 @@ int augtree_prefill_bwd(const augtree_plan_t *pl, const void *q_p, const void *k
   a.dq = dq_p; a.dk_out = nullptr; a.dv_out = nullptr; a.dk_acc = dkp_acc; a.dv_acc = dvp_acc; a.causal_fp32 = 1;
   a.d_segs = pl->d_seg_prefill; a.d_tiles = pl->d_tiles_prefill; a.n_tiles = (long long)pl->tiles_prefill.size() / 2;
   a.dq_sched = &pl->sched[SCHED_PREFILL_DQ]; a.ka = k_p; a.va = v_p; a.a_tok = pl->total_p;
+  a.d_pairs = pl->d_pairs_prefill; a.ds_slots = pl->ds_slots_prefill;
   const Sched &s = pl->sched[SCHED_PREFILL_BWD];
-  r = pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, st) : launch_bwd<64>(pl, s, a, ws, st);
+  r = pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, ws_bytes, st) : launch_bwd<64>(pl, s, a, ws, ws_bytes, st);
   if (r) return r;
   const long long n4 = pl->total_p * (long long)pl->h_kv * pl->head_dim / 4;
   if (dk_p) { cast_bf16_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(dkp_acc, static_cast<__nv_bfloat16 *>(dk_p), n4); ++g_launches; }

@@ -44,6 +44,11 @@ struct BwdParams {
   int kind;                 // schedule index: status[2 + kind] counts finished items
   int test_flags;           // TEST_SKIP_BWD_LOAD: lane 0 never loads the first dO tile of its first item
   int no_own;               // partial-state variant: items inside a sequence (mode 0) are skipped by every role
+  // dS hand-off (null: off): dS^T of every (KV tile, query tile, head) pair is also stored, bf16, as a row-major
+  // [128 keys][128 queries] tile in slot pair_tab[t].x * h_q + head * pair_tab[t].y + (index of the KV tile among
+  // those the query tile sees), for a query-side kernel that then needs neither S nor dP again (dql_kernel)
+  __nv_bfloat16 *ds_out;
+  const int4 *pair_tab;     // per query tile {first slot / h_q, KV tiles seen, prompt KV tiles among them, 0}
 };
 
 constexpr int kBwdThreads = 576;  // 16 element-wise warps, TMA warp, MMA warp
@@ -319,11 +324,20 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const bool key_valid = r < kv_rows;
       bool first = true;
       for (int sg = seg0; sg < seg0 + nseg && ok; ++sg) {
-        const int s_len = p.segs[3 * sg + 1];
+        const int s_len = p.segs[3 * sg + 1], s_tile0 = p.segs[3 * sg + 2];
         const int nqt = (s_len + 127) >> 7;
         const int qt0 = mode ? 0 : (kv_pos0 >> 7);
-        for (int qt = qt0; qt < nqt && ok; ++qt)
-          for (int j = 0; j < rep; ++j, ++T) {
+        for (int qt = qt0; qt < nqt && ok; ++qt) {
+          // hand-off: where this thread's 64 bytes of the pair's dS^T tile go (head j = 0), and the step to the next head
+          __nv_bfloat16 *ds_dst = nullptr;
+          long long ds_step = 0;
+          if (p.ds_out) {
+            const int4 pt = __ldg(p.pair_tab + s_tile0 + qt);
+            const long long slot = (long long)pt.x * p.h_q + (long long)(kvh * rep) * pt.y + (mode ? 0 : pt.z) + (kv_pos0 >> 7);
+            ds_dst = p.ds_out + slot * 16384 + r * 128 + ch * 32;
+            ds_step = (long long)pt.y * 16384;
+          }
+          for (int j = 0; j < rep; ++j, ++T, ds_dst += ds_step) {
             const uint32_t st = T % NST;
             if (first) {  // the item's first pair has no predecessor to pipeline behind
               ok = make_p(T, qt * 128, kv_pos0, mode, key_valid);
@@ -352,6 +366,12 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 dd[i / 2 + 1] = pack_bf16(a1.x, a1.y);
               }
               tmem_st16(tR1 + lane_off + ch * 32, dd);
+              if (p.ds_out) {
+                // hand-off: this thread's 32 values are 64 contiguous bytes of the stored tile, written as two whole
+                // 32-byte sectors (16-byte stores leave half sectors behind and were measured 1.7x slower)
+#pragma unroll
+                for (int i = 0; i < 2; ++i) st_global_v8(ds_dst + 16 * i, dd + 8 * i);
+              }
             }
             tc_wait_st();
             tc_fence_before();
@@ -371,6 +391,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               }
             }
           }
+        }
       }
       if (!ok) break;
       // ---- item epilogue: dV, dK of key row r, columns (D/4)*ch ..

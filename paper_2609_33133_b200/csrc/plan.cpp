@@ -116,6 +116,22 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
   for (int i = 0; i < (int)nb; ++i) add_segment(p->seg_replay, p->tiles_replay, p->cu_r[i], p->branch_len[i]);
   for (int g = 0; g < ng; ++g) add_segment(p->seg_prefill, p->tiles_prefill, p->cu_p[g], p->prompt_len[g]);
 
+  // dS hand-off tables: query tile t of a backward call sees n_t KV tiles (the group's prompt tiles in the replay call,
+  // then the causal tiles of its own sequence); its (head, KV tile) pairs own consecutive 128 x 128 slots of the scratch
+  p->pairs_replay.clear(); p->pairs_prefill.clear();
+  auto add_pairs = [](std::vector<int32_t> &tab, int64_t &slots, int len, int n_prompt_tiles) {
+    for (int t = 0; t < cdiv(len, kTileQ); ++t) {
+      const int n = n_prompt_tiles + t + 1;
+      const int32_t e[4] = {(int32_t)slots, n, n_prompt_tiles, 0};
+      tab.insert(tab.end(), e, e + 4);
+      slots += n;
+    }
+  };
+  p->ds_slots_replay = p->ds_slots_prefill = 0;
+  for (int i = 0; i < (int)nb; ++i)
+    add_pairs(p->pairs_replay, p->ds_slots_replay, p->branch_len[i], cdiv(p->prompt_len[p->branch_group[i]], kTileKV));
+  for (int g = 0; g < ng; ++g) add_pairs(p->pairs_prefill, p->ds_slots_prefill, p->prompt_len[g], 0);
+
   // prompt-KV shards per group: shard = a run of whole KV tiles
   p->group_splits.resize(ng);
   std::vector<int> shard_tiles(ng);
@@ -234,6 +250,9 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
   // backward: row statistics [H_q][tiles][2][128] fp32
   const size_t ntile = std::max(p->tiles_replay.size(), p->tiles_prefill.size()) / 2;
   p->ws_bwd = al(hq * ntile * 2 * kTileQ * 4);
+  // with this much, the key-side kernel also stores dS (bf16, one 128 x 128 tile per pair and head) for the query side
+  const int64_t ds_slots = std::max(p->ds_slots_replay, p->ds_slots_prefill);
+  p->ws_bwd_handoff = ds_slots > 0x3fffffff ? ~(size_t)0 : p->ws_bwd + al((size_t)ds_slots * hq * (size_t)(kTileQ * kTileKV * 2));
   (void)tmax; (void)dd;
   return AUGTREE_OK;
 }

@@ -48,14 +48,19 @@ struct augtree_plan {
   std::vector<int32_t> cu_p, cu_b, cu_r, branch_group, group_splits;
   std::vector<int32_t> seg_replay, seg_prefill;    // [n][3] {first query token, length, first tile index}
   std::vector<int32_t> tiles_replay, tiles_prefill;  // [n_tiles][2] {first token, rows}: 128-row query tiles per segment
+  // dS hand-off of the backward pass: per query tile {first slot / heads, KV tiles it sees, prompt KV tiles among them, 0}
+  std::vector<int32_t> pairs_replay, pairs_prefill;
+  int64_t ds_slots_replay = 0, ds_slots_prefill = 0;  // (KV tile, query tile) pairs per head of each backward call
   augtree::Sched sched[augtree::SCHED_COUNT];
   int32_t *d_seg_replay = nullptr, *d_seg_prefill = nullptr, *d_branch_group = nullptr, *d_group_splits = nullptr;
   int32_t *d_cu_r = nullptr;
   int32_t *d_tiles_replay = nullptr, *d_tiles_prefill = nullptr;
+  int32_t *d_pairs_replay = nullptr, *d_pairs_prefill = nullptr;
   int *d_status = nullptr;  // [kStatusInts]: status, detail, then the items each schedule's kernel has finished
   mutable std::atomic<long long> launched_items[augtree::SCHED_COUNT] = {};  // items handed to launches so far
   augtree::Timing *timing = nullptr;  // optional CUDA-event timing of the tile kernels
   size_t ws_fwd = 0, ws_bwd = 0;
+  size_t ws_bwd_handoff = 0;  // backward scratch at which the key-side kernel hands dS to the query-side kernel
 };
 
 namespace augtree {

@@ -20,11 +20,11 @@ GRADS = ["dq_p", "dk_p", "dv_p", "dq_r", "dk_r", "dv_r"]
 U_BF16 = 2.0 ** -8                            # unit roundoff of bf16, round to nearest (8 significant bits)
 
 
-def run_gpu(B, w, t_cpu, kv_splits=0, n_lanes=0, flags=0):
+def run_gpu(B, w, t_cpu, kv_splits=0, n_lanes=0, flags=0, handoff_limit=None):
     plan = B.Plan(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, device=0, kv_splits=kv_splits,
                   n_lanes=n_lanes, flags=flags)
     t = {k: v.cuda() for k, v in t_cpu.items()}
-    out = B.alloc_outputs(plan)
+    out = B.alloc_outputs(plan) if handoff_limit is None else B.alloc_outputs(plan, handoff_limit=handoff_limit)
     B.run_forward_backward(plan, t, out)
     torch.cuda.synchronize()
     status = plan.device_status()

@@ -195,3 +195,19 @@ def test_assign_grid_rejects_bad_arguments(binding):
         binding.assign_grid([1, 2], None, 1, 1, cell_cap=3)  # a limit needs sizes
     assert e.value.code == -1
     assert binding.assign_grid([], None, 2, 2) == ([], [], 0, True)
+
+
+def test_handoff_scratch_counts_every_visible_tile_pair(binding):
+    """Backward hand-off scratch = row statistics + one 32 KB dS tile per (query tile, visible KV tile, query head) of the
+    larger backward call, counted here from the definition of visibility (Eq. 1)."""
+    B = binding
+    cdiv = lambda a, b: -(-a // b)
+    for pl, bl, hq, hkv, d in [([700], [[300, 150, 420]], 8, 2, 128), ([129, 1000], [[1, 257], [640, 64, 130, 127]], 4, 4, 64),
+                               ([8192], [[2048] * 8], 28, 4, 128), ([300], [[]], 4, 2, 64)]:
+        plan = B.Plan(pl, bl, hq, hkv, d, device=None, n_lanes=8)
+        replay = sum(cdiv(P, 128) * cdiv(r, 128) + cdiv(r, 128) * (cdiv(r, 128) + 1) // 2 for P, rs in zip(pl, bl) for r in rs)
+        prefill = sum(cdiv(P, 128) * (cdiv(P, 128) + 1) // 2 for P in pl)
+        extra = plan.ws_bwd_handoff_bytes - plan.ws_bwd_bytes
+        assert extra == max(replay, prefill) * hq * 128 * 128 * 2, (pl, bl)
+        assert plan.workspace_bytes(0) == max(plan.ws_fwd_bytes, plan.ws_bwd_bytes, 256)
+        assert plan.workspace_bytes(1 << 50) >= plan.ws_bwd_handoff_bytes
