@@ -55,7 +55,7 @@ extern "C" {
 typedef enum {
   AUGTREE_OK = 0,
   AUGTREE_ERR_INVALID_ARG = -1, /* null pointer, non-positive length, bad struct size   */
-  AUGTREE_ERR_UNSUPPORTED = -2, /* head_dim not 64/128, h_q % h_kv != 0, sizes too big  */
+  AUGTREE_ERR_UNSUPPORTED = -2, /* head_dim unsupported, h_q % h_kv != 0, sizes too big */
   AUGTREE_ERR_WORKSPACE = -3,   /* workspace pointer null or too small                  */
   AUGTREE_ERR_CUDA = -4,        /* a CUDA runtime or driver call failed                 */
   AUGTREE_ERR_TIMEOUT = -5,     /* a device-side wait gave up (status word)             */
@@ -98,7 +98,7 @@ typedef struct {
   const int32_t *prompt_len;  /* [n_groups]                                       (host) */
   const int32_t *n_branches;  /* [n_groups]                                       (host) */
   const int32_t *branch_len;  /* [sum n_branches], group-major                    (host) */
-  int32_t h_q, h_kv, head_dim;/* head_dim in {64, 128}                                   */
+  int32_t h_q, h_kv, head_dim;/* multiple of 8, 8..128; tiles are 64 or 128 wide      */
   float softmax_scale;        /* 0 => 1/sqrt(head_dim)  (Sec. 2.2)                       */
   uint32_t flags;
   int32_t n_lanes;            /* replay lanes = persistent CTAs; 0 => SM count of device */

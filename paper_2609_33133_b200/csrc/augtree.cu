@@ -131,20 +131,20 @@ int launch_fwd(const augtree_plan *pl, const Sched &s, const void *q, long long 
     if (blocks > 1 && cudaMemsetAsync(kmax2, 0, (size_t)pl->h_kv * sizeof(unsigned int), st) != cudaSuccess) return AUGTREE_ERR_CUDA;
     key_norm_kernel<D><<<dim3(blocks, (unsigned)pl->h_kv), 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(ka), a_tok,
                                                                        static_cast<const __nv_bfloat16 *>(kb), same ? 0 : b_tok,
-                                                                       pl->h_kv, kmax2);
+                                                                       pl->h_kv, pl->head_dim, kmax2);
     ++g_launches;
   }
   CUtensorMap mq, mka, mva, mkb, mvb;
   int r;
-  if ((r = make_map(&mq, q, q_tok, pl->h_q, D))) return r;
-  if ((r = make_map(&mka, ka, a_tok, pl->h_kv, D))) return r;
-  if ((r = make_map(&mva, va, a_tok, pl->h_kv, D))) return r;
-  if ((r = make_map(&mkb, kb, b_tok, pl->h_kv, D))) return r;
-  if ((r = make_map(&mvb, vb, b_tok, pl->h_kv, D))) return r;
+  if ((r = make_map(&mq, q, q_tok, pl->h_q, pl->head_dim))) return r;
+  if ((r = make_map(&mka, ka, a_tok, pl->h_kv, pl->head_dim))) return r;
+  if ((r = make_map(&mva, va, a_tok, pl->h_kv, pl->head_dim))) return r;
+  if ((r = make_map(&mkb, kb, b_tok, pl->h_kv, pl->head_dim))) return r;
+  if ((r = make_map(&mvb, vb, b_tok, pl->h_kv, pl->head_dim))) return r;
   FwdParams p;
   p.items = s.d_items; p.lane_ptr = s.d_lane_ptr;
   p.o = static_cast<__nv_bfloat16 *>(o); p.lse = lse; p.part_o = part_o; p.part_lse = part_lse;
-  p.n_tok = q_tok; p.h_q = pl->h_q; p.scale_log2 = pl->scale * 1.4426950408889634f; p.status = pl->d_status;
+  p.n_tok = q_tok; p.h_q = pl->h_q; p.d = pl->head_dim; p.scale_log2 = pl->scale * 1.4426950408889634f; p.status = pl->d_status;
   p.kmax2 = reinterpret_cast<const float *>(kmax2);
   const int kind = (int)(&s - pl->sched);
   p.wait_budget = wait_budget(pl); p.kind = kind;
@@ -191,22 +191,22 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
   {
     const dim3 grid((unsigned)a.n_tiles, (unsigned)pl->h_q);
     bwd_preprocess_kernel<D><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(a.o), static_cast<const __nv_bfloat16 *>(a.d_o),
-                                                   a.lse, a.d_tiles, stats, a.q_tok, a.n_tiles, pl->h_q, pl->scale);
+                                                   a.lse, a.d_tiles, stats, a.q_tok, a.n_tiles, pl->h_q, pl->head_dim, pl->scale);
     ++g_launches;
   }
   CUtensorMap mq, mdo, mk0, mv0, mk1, mv1;
   int r;
-  if ((r = make_map(&mq, a.q, a.q_tok, pl->h_q, D))) return r;
-  if ((r = make_map(&mdo, a.d_o, a.q_tok, pl->h_q, D))) return r;
-  if ((r = make_map(&mk0, a.k0, a.kv0_tok, pl->h_kv, D))) return r;
-  if ((r = make_map(&mv0, a.v0, a.kv0_tok, pl->h_kv, D))) return r;
-  if ((r = make_map(&mk1, a.k1, a.kv1_tok, pl->h_kv, D))) return r;
-  if ((r = make_map(&mv1, a.v1, a.kv1_tok, pl->h_kv, D))) return r;
+  if ((r = make_map(&mq, a.q, a.q_tok, pl->h_q, pl->head_dim))) return r;
+  if ((r = make_map(&mdo, a.d_o, a.q_tok, pl->h_q, pl->head_dim))) return r;
+  if ((r = make_map(&mk0, a.k0, a.kv0_tok, pl->h_kv, pl->head_dim))) return r;
+  if ((r = make_map(&mv0, a.v0, a.kv0_tok, pl->h_kv, pl->head_dim))) return r;
+  if ((r = make_map(&mk1, a.k1, a.kv1_tok, pl->h_kv, pl->head_dim))) return r;
+  if ((r = make_map(&mv1, a.v1, a.kv1_tok, pl->h_kv, pl->head_dim))) return r;
   if (s.n_items() > 0) {
     BwdParams p;
     p.items = s.d_items; p.lane_ptr = s.d_lane_ptr; p.segs = a.d_segs; p.stats = stats;
     p.dk_out = static_cast<__nv_bfloat16 *>(a.dk_out); p.dv_out = static_cast<__nv_bfloat16 *>(a.dv_out);
-    p.dk_acc = a.dk_acc; p.dv_acc = a.dv_acc; p.n_tiles = a.n_tiles; p.h_q = pl->h_q; p.h_kv = pl->h_kv;
+    p.dk_acc = a.dk_acc; p.dv_acc = a.dv_acc; p.n_tiles = a.n_tiles; p.h_q = pl->h_q; p.h_kv = pl->h_kv; p.d = pl->head_dim;
     p.causal_fp32 = a.causal_fp32; p.scale = pl->scale; p.scale_log2 = pl->scale * 1.4426950408889634f;
     p.status = pl->d_status;
     const int kind = (int)(&s - pl->sched);
@@ -229,10 +229,10 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
   if (handoff) {
     CUtensorMap mds, mka;
     if ((r = make_ds_map(&mds, ds, a.ds_slots * pl->h_q))) return r;
-    if ((r = make_map(&mka, a.ka, a.a_tok, pl->h_kv, D))) return r;
+    if ((r = make_map(&mka, a.ka, a.a_tok, pl->h_kv, pl->head_dim))) return r;
     DqlParams p;
     p.items = a.dq_sched->d_items; p.lane_ptr = a.dq_sched->d_lane_ptr; p.pair_tab = reinterpret_cast<const int4 *>(a.d_pairs);
-    p.dq = static_cast<__nv_bfloat16 *>(a.dq); p.dq_f32 = a.dq_f32; p.h_q = pl->h_q; p.no_own = a.no_own;
+    p.dq = static_cast<__nv_bfloat16 *>(a.dq); p.dq_f32 = a.dq_f32; p.h_q = pl->h_q; p.d = pl->head_dim; p.no_own = a.no_own;
     p.status = pl->d_status;
     const int kind = (int)(a.dq_sched - pl->sched);
     p.wait_budget = wait_budget(pl); p.kind = kind;
@@ -243,11 +243,11 @@ int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *w
     ++g_launches;
   } else if (a.dq_sched->n_items() > 0) {
     CUtensorMap mka, mva;
-    if ((r = make_map(&mka, a.ka, a.a_tok, pl->h_kv, D))) return r;
-    if ((r = make_map(&mva, a.va, a.a_tok, pl->h_kv, D))) return r;
+    if ((r = make_map(&mka, a.ka, a.a_tok, pl->h_kv, pl->head_dim))) return r;
+    if ((r = make_map(&mva, a.va, a.a_tok, pl->h_kv, pl->head_dim))) return r;
     DqParams p;
     p.items = a.dq_sched->d_items; p.lane_ptr = a.dq_sched->d_lane_ptr; p.stats = stats;
-    p.dq = static_cast<__nv_bfloat16 *>(a.dq); p.n_tiles = a.n_tiles; p.h_q = pl->h_q;
+    p.dq = static_cast<__nv_bfloat16 *>(a.dq); p.n_tiles = a.n_tiles; p.h_q = pl->h_q; p.d = pl->head_dim;
     p.scale = pl->scale; p.scale_log2 = pl->scale * 1.4426950408889634f; p.status = pl->d_status;
     const int kind = (int)(a.dq_sched - pl->sched);
     p.wait_budget = wait_budget(pl); p.kind = kind;
@@ -334,7 +334,7 @@ int augtree_plan_create(const augtree_desc_t *desc, int device, augtree_plan_t *
     int prev = 0;
     cudaGetDevice(&prev);
     r = cudaSetDevice(device) == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
-    if (!r) r = pl->head_dim == 128 ? set_kernel_attributes<128>() : set_kernel_attributes<64>();
+    if (!r) r = pl->head_dim > 64 ? set_kernel_attributes<128>() : set_kernel_attributes<64>();
     try {
       for (int k = 0; k < SCHED_COUNT && !r; ++k)
         r = upload_sched(pl->sched[k], pl->n_lanes, k == SCHED_REPLAY_FWD && (pl->flags & AUGTREE_FLAG_TEST_DROP_ITEM));
@@ -435,7 +435,7 @@ int augtree_prefill_fwd(const augtree_plan_t *pl, const void *q_p, const void *k
   if (!ws || ws_bytes < kFwdHeaderBytes || !aligned16(ws)) return AUGTREE_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Sched &s = pl->sched[SCHED_PREFILL_FWD];
-  if (pl->head_dim == 128)
+  if (pl->head_dim > 64)
     return launch_fwd<128>(pl, s, q_p, pl->total_p, k_p, v_p, pl->total_p, k_p, v_p, pl->total_p, o_p, lse_p, nullptr, nullptr, ws, st);
   return launch_fwd<64>(pl, s, q_p, pl->total_p, k_p, v_p, pl->total_p, k_p, v_p, pl->total_p, o_p, lse_p, nullptr, nullptr, ws, st);
 }
@@ -457,7 +457,7 @@ int augtree_replay_fwd(const augtree_plan_t *pl, const void *q_r, const void *k_
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Sched &s = pl->sched[SCHED_REPLAY_FWD];
-  if (pl->head_dim == 128)
+  if (pl->head_dim > 64)
     r = launch_fwd<128>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, o_r, lse_r, part_o, part_lse, ws, st);
   else
     r = launch_fwd<64>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, o_r, lse_r, part_o, part_lse, ws, st);
@@ -466,12 +466,12 @@ int augtree_replay_fwd(const augtree_plan_t *pl, const void *q_r, const void *k_
   // merge kernel only touches tokens whose group has more than one shard
   const long long warps = pl->total_r * (long long)pl->h_q;
   const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
-  if (pl->head_dim == 128)
+  if (pl->head_dim > 64)
     combine_kernel<128><<<blocks, 256, 0, st>>>(part_o, part_lse, pl->d_cu_r, pl->d_branch_group, pl->d_group_splits,
-                                                pl->n_branches, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q);
+                                                pl->n_branches, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q, pl->head_dim);
   else
     combine_kernel<64><<<blocks, 256, 0, st>>>(part_o, part_lse, pl->d_cu_r, pl->d_branch_group, pl->d_group_splits,
-                                               pl->n_branches, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q);
+                                               pl->n_branches, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q, pl->head_dim);
   ++g_launches;
   return cudaGetLastError() == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
 }
@@ -518,7 +518,7 @@ int augtree_replay_fwd_state(const augtree_plan_t *pl, const void *q_r, const vo
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Sched &s = pl->sched[SCHED_REPLAY_FWD];
   const int mode = STATE_OUT | (include_own ? 0 : STATE_NO_OWN);
-  if (pl->head_dim == 128)
+  if (pl->head_dim > 64)
     return launch_fwd<128>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, nullptr, nullptr, state_o, state_lse, ws, st, mode);
   return launch_fwd<64>(pl, s, q_r, pl->total_r, k_p, v_p, pl->total_p, k_r, v_r, pl->total_r, nullptr, nullptr, state_o, state_lse, ws, st, mode);
 }
@@ -538,10 +538,10 @@ int augtree_merge_states(const augtree_plan_t *pl, int n_states, const float *co
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const long long warps = pl->total_r * (long long)pl->h_q;
   const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
-  if (pl->head_dim == 128)
-    merge_states_kernel<128><<<blocks, 256, 0, st>>>(sp, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q);
+  if (pl->head_dim > 64)
+    merge_states_kernel<128><<<blocks, 256, 0, st>>>(sp, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q, pl->head_dim);
   else
-    merge_states_kernel<64><<<blocks, 256, 0, st>>>(sp, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q);
+    merge_states_kernel<64><<<blocks, 256, 0, st>>>(sp, static_cast<__nv_bfloat16 *>(o_r), lse_r, pl->total_r, pl->h_q, pl->head_dim);
   ++g_launches;
   return cudaGetLastError() == cudaSuccess ? AUGTREE_OK : AUGTREE_ERR_CUDA;
 }
@@ -574,7 +574,7 @@ int augtree_replay_bwd_state(const augtree_plan_t *pl, const void *q_r, const vo
   a.d_pairs = pl->d_pairs_replay; a.ds_slots = pl->ds_slots_replay;
   a.no_own = include_own ? 0 : 1; a.dq_f32 = dq_part;
   const Sched &s = pl->sched[SCHED_REPLAY_BWD];
-  return pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, ws_bytes, st) : launch_bwd<64>(pl, s, a, ws, ws_bytes, st);
+  return pl->head_dim > 64 ? launch_bwd<128>(pl, s, a, ws, ws_bytes, st) : launch_bwd<64>(pl, s, a, ws, ws_bytes, st);
 }
 
 int augtree_replay_bwd(const augtree_plan_t *pl, const void *q_r, const void *k_r, const void *v_r, const void *k_p,
@@ -603,7 +603,7 @@ int augtree_replay_bwd(const augtree_plan_t *pl, const void *q_r, const void *k_
   a.dq_sched = &pl->sched[SCHED_REPLAY_DQ]; a.ka = k_p; a.va = v_p; a.a_tok = pl->total_p;
   a.d_pairs = pl->d_pairs_replay; a.ds_slots = pl->ds_slots_replay;
   const Sched &s = pl->sched[SCHED_REPLAY_BWD];
-  return pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, ws_bytes, st) : launch_bwd<64>(pl, s, a, ws, ws_bytes, st);
+  return pl->head_dim > 64 ? launch_bwd<128>(pl, s, a, ws, ws_bytes, st) : launch_bwd<64>(pl, s, a, ws, ws_bytes, st);
 }
 
 int augtree_prefill_bwd(const augtree_plan_t *pl, const void *q_p, const void *k_p, const void *v_p, const void *o_p,
@@ -625,7 +625,7 @@ int augtree_prefill_bwd(const augtree_plan_t *pl, const void *q_p, const void *k
   a.dq_sched = &pl->sched[SCHED_PREFILL_DQ]; a.ka = k_p; a.va = v_p; a.a_tok = pl->total_p;
   a.d_pairs = pl->d_pairs_prefill; a.ds_slots = pl->ds_slots_prefill;
   const Sched &s = pl->sched[SCHED_PREFILL_BWD];
-  r = pl->head_dim == 128 ? launch_bwd<128>(pl, s, a, ws, ws_bytes, st) : launch_bwd<64>(pl, s, a, ws, ws_bytes, st);
+  r = pl->head_dim > 64 ? launch_bwd<128>(pl, s, a, ws, ws_bytes, st) : launch_bwd<64>(pl, s, a, ws, ws_bytes, st);
   if (r) return r;
   const long long n4 = pl->total_p * (long long)pl->h_kv * pl->head_dim / 4;
   if (dk_p) { cast_bf16_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(dkp_acc, static_cast<__nv_bfloat16 *>(dk_p), n4); ++g_launches; }

@@ -37,6 +37,7 @@ struct BwdParams {
   float *dk_acc, *dv_acc;   // fp32 [prompt tokens, h_kv, D]: mode-1 items, and mode-0 items when causal_fp32 != 0
   long long n_tiles;        // query tiles in the stats table
   int h_q, h_kv;
+  int d;                    // head dimension of the tensors (<= D; columns d.. of every tile read as zero)
   int causal_fp32;
   float scale, scale_log2;
   int *status;
@@ -410,19 +411,20 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         tc_wait_ld();
         if (key_valid) {
           if (to_fp32) {
-            float4 *dst = reinterpret_cast<float4 *>((which ? p.dk_acc : p.dv_acc) + krow * D + col0);
+            float4 *dst = reinterpret_cast<float4 *>((which ? p.dk_acc : p.dv_acc) + krow * p.d + col0);
 #pragma unroll
             for (int i = 0; i < QUART / 4; ++i) {
+              if (col0 + 4 * i >= p.d) break;  // padding columns
               float4 a = dst[i];
               a.x += __uint_as_float(v[4 * i]); a.y += __uint_as_float(v[4 * i + 1]);
               a.z += __uint_as_float(v[4 * i + 2]); a.w += __uint_as_float(v[4 * i + 3]);
               dst[i] = a;
             }
           } else {
-            uint4 *dst = reinterpret_cast<uint4 *>((which ? p.dk_out : p.dv_out) + krow * D + col0);
+            uint4 *dst = reinterpret_cast<uint4 *>((which ? p.dk_out : p.dv_out) + krow * p.d + col0);
 #pragma unroll
             for (int i = 0; i < QUART / 8; ++i)
-              dst[i] = make_uint4(pack_bf16(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
+              if (col0 + 8 * i < p.d) dst[i] = make_uint4(pack_bf16(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
                                   pack_bf16(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
                                   pack_bf16(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
                                   pack_bf16(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
@@ -452,7 +454,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 // stats[head][tile][1][i] = -scale * sum_d dO * O (0 past the end).  One warp per 16 rows.
 template <int D>
 __global__ void bwd_preprocess_kernel(const __nv_bfloat16 *o, const __nv_bfloat16 *d_o, const float *lse, const int32_t *tiles,
-                                      float *stats, long long n_tok, long long n_tiles, int h_q, float scale) {
+                                      float *stats, long long n_tok, long long n_tiles, int h_q, int d, float scale) {
   const int tile = blockIdx.x, head = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tok0 = tiles[2 * tile], rows = tiles[2 * tile + 1];
@@ -466,8 +468,8 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16 *o, const __nv_bfloat1
   for (int ps = 0; ps < PASSES; ++ps) {
     const int i = warp * 16 + ps * RPP + sub;
     vo[ps] = make_uint4(0, 0, 0, 0); vd[ps] = make_uint4(0, 0, 0, 0);
-    if (i < rows) {
-      const long long w = (((long long)tok0 + i) * h_q + head) * D + part * 8;
+    if (i < rows && part * 8 < d) {
+      const long long w = (((long long)tok0 + i) * h_q + head) * d + part * 8;
       vo[ps] = *reinterpret_cast<const uint4 *>(o + w);
       vd[ps] = *reinterpret_cast<const uint4 *>(d_o + w);
     }

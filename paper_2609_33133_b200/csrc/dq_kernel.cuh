@@ -31,6 +31,7 @@ struct DqParams {
   __nv_bfloat16 *dq;        // [query tokens, h_q, D]
   long long n_tiles;
   int h_q;
+  int d;                    // head dimension of the tensors (<= D)
   float scale, scale_log2;
   int *status;
   long long wait_budget;    // clocks a wait may take before the kernel gives up
@@ -321,22 +322,22 @@ dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       tc_fence_after();
       {
         constexpr int HALF = D / 2;
-        __nv_bfloat16 *dst_row = p.dq + (((long long)q_tok0 + r) * p.h_q + head) * D + ch * HALF;
+        __nv_bfloat16 *dst_row = p.dq + (((long long)q_tok0 + r) * p.h_q + head) * p.d + ch * HALF;
 #pragma unroll
         for (int c = 0; c < HALF / 32; ++c) {
           uint32_t v[32];
           tmem_ld32(tDQ + lane_off + ch * HALF + c * 32, v);
           tc_wait_ld();
           if (r < q_rows && p.dq_f32) {
-            float4 *dst = reinterpret_cast<float4 *>(p.dq_f32 + (((long long)q_tok0 + r) * p.h_q + head) * D + ch * HALF + c * 32);
+            float4 *dst = reinterpret_cast<float4 *>(p.dq_f32 + (((long long)q_tok0 + r) * p.h_q + head) * p.d + ch * HALF + c * 32);
 #pragma unroll
             for (int e = 0; e < 8; ++e)
-              dst[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]), __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
+              if (ch * HALF + c * 32 + 4 * e < p.d) dst[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]), __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
           } else if (r < q_rows) {
             uint4 *dst = reinterpret_cast<uint4 *>(dst_row + c * 32);
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-              dst[e] = make_uint4(pack_bf16(__uint_as_float(v[8 * e]), __uint_as_float(v[8 * e + 1])),
+              if (ch * HALF + c * 32 + 8 * e < p.d) dst[e] = make_uint4(pack_bf16(__uint_as_float(v[8 * e]), __uint_as_float(v[8 * e + 1])),
                                   pack_bf16(__uint_as_float(v[8 * e + 2]), __uint_as_float(v[8 * e + 3])),
                                   pack_bf16(__uint_as_float(v[8 * e + 4]), __uint_as_float(v[8 * e + 5])),
                                   pack_bf16(__uint_as_float(v[8 * e + 6]), __uint_as_float(v[8 * e + 7])));

@@ -22,6 +22,7 @@ struct DqlParams {
   __nv_bfloat16 *dq;        // [query tokens, h_q, D]
   float *dq_f32;            // partial-state variant: dQ is written here in fp32
   int h_q;
+  int d;                    // head dimension of the tensors (<= D)
   int no_own;               // partial-state variant: the causal range of the query's own sequence is left out
   int *status;
   long long wait_budget;
@@ -151,7 +152,7 @@ dql_kernel(const __grid_constant__ CUtensorMap tm_ds, const __grid_constant__ CU
       ok = mbar_wait(bar_acc_full + 8 * buf, (ic >> 1) & 1, ab, WAIT_DQL_ACC_FULL);
       if (!ok) break;
       tc_fence_after();
-      const long long row_off = (((long long)q_tok0 + r) * p.h_q + head) * D;
+      const long long row_off = (((long long)q_tok0 + r) * p.h_q + head) * p.d;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t v[32];
@@ -161,12 +162,12 @@ dql_kernel(const __grid_constant__ CUtensorMap tm_ds, const __grid_constant__ CU
           float4 *dst = reinterpret_cast<float4 *>(p.dq_f32 + row_off + c * 32);
 #pragma unroll
           for (int e = 0; e < 8; ++e)
-            dst[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]), __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
+            if (c * 32 + 4 * e < p.d) dst[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]), __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
         } else if (r < q_rows) {
           uint4 *dst = reinterpret_cast<uint4 *>(p.dq + row_off + c * 32);
 #pragma unroll
           for (int e = 0; e < 4; ++e)
-            dst[e] = make_uint4(pack_bf16(__uint_as_float(v[8 * e]), __uint_as_float(v[8 * e + 1])),
+            if (c * 32 + 8 * e < p.d) dst[e] = make_uint4(pack_bf16(__uint_as_float(v[8 * e]), __uint_as_float(v[8 * e + 1])),
                                 pack_bf16(__uint_as_float(v[8 * e + 2]), __uint_as_float(v[8 * e + 3])),
                                 pack_bf16(__uint_as_float(v[8 * e + 4]), __uint_as_float(v[8 * e + 5])),
                                 pack_bf16(__uint_as_float(v[8 * e + 6]), __uint_as_float(v[8 * e + 7])));

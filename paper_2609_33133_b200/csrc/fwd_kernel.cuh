@@ -31,6 +31,7 @@ struct FwdParams {
   float *part_lse;          // [splits, h_q, tokens]
   long long n_tok;          // tokens in the query tensor
   int h_q;
+  int d;                    // head dimension of the tensors (<= D; D is the padded tile width, columns d.. read as zero)
   float scale_log2;         // softmax scale * log2(e)
   const float *kmax2;       // [h_kv] largest squared key norm of the call's K tensors (key_norm_kernel)
   int *status;
@@ -460,15 +461,16 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int col = c * 32 + 8 * i + cq;
+            if (col >= p.d) continue;  // padding columns of a head dimension below D
             if (n_splits == 1) {
-              if (validA) *reinterpret_cast<uint32_t *>(p.o + (tokA * p.h_q + head) * D + col) =
+              if (validA) *reinterpret_cast<uint32_t *>(p.o + (tokA * p.h_q + head) * p.d + col) =
                   pack_bf16(__uint_as_float(o[4 * i]) * invA, __uint_as_float(o[4 * i + 1]) * invA);
-              if (validB) *reinterpret_cast<uint32_t *>(p.o + (tokB * p.h_q + head) * D + col) =
+              if (validB) *reinterpret_cast<uint32_t *>(p.o + (tokB * p.h_q + head) * p.d + col) =
                   pack_bf16(__uint_as_float(o[4 * i + 2]) * invB, __uint_as_float(o[4 * i + 3]) * invB);
             } else {
-              if (validA) *reinterpret_cast<float2 *>(p.part_o + (((long long)split * p.n_tok + tokA) * p.h_q + head) * D + col) =
+              if (validA) *reinterpret_cast<float2 *>(p.part_o + (((long long)split * p.n_tok + tokA) * p.h_q + head) * p.d + col) =
                   make_float2(__uint_as_float(o[4 * i]) * invA, __uint_as_float(o[4 * i + 1]) * invA);
-              if (validB) *reinterpret_cast<float2 *>(p.part_o + (((long long)split * p.n_tok + tokB) * p.h_q + head) * D + col) =
+              if (validB) *reinterpret_cast<float2 *>(p.part_o + (((long long)split * p.n_tok + tokB) * p.h_q + head) * p.d + col) =
                   make_float2(__uint_as_float(o[4 * i + 2]) * invB, __uint_as_float(o[4 * i + 3]) * invB);
             }
           }
@@ -513,7 +515,7 @@ struct StatePtrs {
   int n;
 };
 template <int D>
-__global__ void merge_states_kernel(const StatePtrs sp, __nv_bfloat16 *o, float *lse, long long n_tok, int h_q) {
+__global__ void merge_states_kernel(const StatePtrs sp, __nv_bfloat16 *o, float *lse, long long n_tok, int h_q, int d) {
   const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (w >= n_tok * h_q) return;
@@ -530,15 +532,17 @@ __global__ void merge_states_kernel(const StatePtrs sp, __nv_bfloat16 *o, float 
   for (int i = 0; i < PER; ++i) acc[i] = 0.f;
   for (int s = 0; s < sp.n; ++s) {
     const float wgt = __expf(sp.lse[s][(long long)head * n_tok + tok] - ref) / den;
-    const float *src = sp.o[s] + (tok * h_q + head) * D + lane * PER;
-    if (wgt > 0.f) {
+    const float *src = sp.o[s] + (tok * h_q + head) * d + lane * PER;
+    if (wgt > 0.f && lane * PER < d) {   // (d is a multiple of 8, PER of 2 or 4: a lane is inside or outside as a whole)
 #pragma unroll
       for (int i = 0; i < PER; ++i) acc[i] += wgt * src[i];
     }
   }
-  __nv_bfloat16 *dst = o + (tok * h_q + head) * D + lane * PER;
+  __nv_bfloat16 *dst = o + (tok * h_q + head) * d + lane * PER;
+  if (lane * PER < d) {
 #pragma unroll
-  for (int i = 0; i < PER; ++i) dst[i] = __float2bfloat16(acc[i]);
+    for (int i = 0; i < PER; ++i) dst[i] = __float2bfloat16(acc[i]);
+  }
   if (lane == 0) lse[(long long)head * n_tok + tok] = ref + __logf(den);
 }
 
@@ -549,7 +553,7 @@ __global__ void merge_states_kernel(const StatePtrs sp, __nv_bfloat16 *o, float 
 // Feeds the score bound that lets the tile kernel skip row maxima; HBM-bound, a few microseconds.
 template <int D>
 __global__ void key_norm_kernel(const __nv_bfloat16 *ka, long long a_tok, const __nv_bfloat16 *kb, long long b_tok, int h_kv,
-                                unsigned int *out) {
+                                int d, unsigned int *out) {
   constexpr int LPR = D / 8, RPP = 32 / LPR;   // 16-byte loads: lanes per (token, head) row, rows per warp pass
   const int lane = threadIdx.x & 31, sub = lane / LPR, part = lane % LPR;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5, n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -561,8 +565,8 @@ __global__ void key_norm_kernel(const __nv_bfloat16 *ka, long long a_tok, const 
     for (long long t0 = warp * RPP; t0 < n; t0 += n_warps * RPP) {
       const long long t = t0 + sub;
       float acc = 0.f;
-      if (t < n) {
-        const uint4 x = *reinterpret_cast<const uint4 *>(k + (t * h_kv + head) * D + part * 8);
+      if (t < n && part * 8 < d) {
+        const uint4 x = *reinterpret_cast<const uint4 *>(k + (t * h_kv + head) * d + part * 8);
         const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -592,7 +596,7 @@ __global__ void key_norm_kernel(const __nv_bfloat16 *ka, long long a_tok, const 
 template <int D>
 __global__ void combine_kernel(const float *part_o, const float *part_lse, const int32_t *cu_r, const int32_t *branch_group,
                                const int32_t *group_splits, int n_branches, __nv_bfloat16 *o, float *lse,
-                               long long n_tok, int h_q) {
+                               long long n_tok, int h_q, int d) {
   const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (w >= n_tok * h_q) return;
@@ -612,13 +616,17 @@ __global__ void combine_kernel(const float *part_o, const float *part_lse, const
   for (int i = 0; i < PER; ++i) acc[i] = 0.f;
   for (int s = 0; s < ns; ++s) {
     const float wgt = __expf(part_lse[((long long)s * h_q + head) * n_tok + tok] - mx) / den;
-    const float *src = part_o + (((long long)s * n_tok + tok) * h_q + head) * D + lane * PER;
+    const float *src = part_o + (((long long)s * n_tok + tok) * h_q + head) * d + lane * PER;
+    if (lane * PER < d) {
 #pragma unroll
-    for (int i = 0; i < PER; ++i) acc[i] += wgt * src[i];
+      for (int i = 0; i < PER; ++i) acc[i] += wgt * src[i];
+    }
   }
-  __nv_bfloat16 *dst = o + (tok * h_q + head) * D + lane * PER;
+  __nv_bfloat16 *dst = o + (tok * h_q + head) * d + lane * PER;
+  if (lane * PER < d) {
 #pragma unroll
-  for (int i = 0; i < PER; ++i) dst[i] = __float2bfloat16(acc[i]);
+    for (int i = 0; i < PER; ++i) dst[i] = __float2bfloat16(acc[i]);
+  }
   if (lane == 0) lse[(long long)head * n_tok + tok] = mx + __logf(den);
 }
 

@@ -65,7 +65,8 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
   if (d->n_groups < 1 || !d->prompt_len || !d->n_branches) return AUGTREE_ERR_INVALID_ARG;
   if (d->h_q < 1 || d->h_kv < 1 || d->n_lanes < 0 || d->kv_splits < 0) return AUGTREE_ERR_INVALID_ARG;
   if (d->h_q % d->h_kv != 0) return AUGTREE_ERR_UNSUPPORTED;
-  if (d->head_dim != 64 && d->head_dim != 128) return AUGTREE_ERR_UNSUPPORTED;
+  // tiles are 64 or 128 columns wide; a head dimension below that is padded with zero columns by the tensor maps
+  if (d->head_dim < 8 || d->head_dim > 128 || d->head_dim % 8 != 0) return AUGTREE_ERR_UNSUPPORTED;
   if (!(d->softmax_scale >= 0.f) || std::isinf(d->softmax_scale)) return AUGTREE_ERR_INVALID_ARG;
 
   p->n_groups = d->n_groups;

@@ -137,12 +137,14 @@ def _guarded(shape, dtype, fill):
     return raw, view, n
 
 
-@pytest.mark.parametrize("case", ["ragged", "sharded", "d64"])
+@pytest.mark.parametrize("case", ["ragged", "sharded", "d64", "d96-sharded", "d40"])
 def test_guard_bands_around_outputs_stay_untouched(B, case):
     w, splits = {
         "ragged": (wl.Workload("canary-ragged", [300, 1, 129], [[5, 130, 257], [1], [64, 200]], 4, 2, 128, 12), 0),
         "sharded": (wl.Workload("canary-sharded", [1100, 200], [[130, 64], [257]], 4, 2, 128, 21), 3),
         "d64": (wl.Workload("canary-d64", [77, 513], [[1, 129], [300]], 6, 2, 64, 13), 0),
+        "d96-sharded": (wl.Workload("canary-d96", [600, 129], [[130, 257], [64]], 4, 2, 96, 14), 2),   # padded tiles
+        "d40": (wl.Workload("canary-d40", [300], [[5, 130]], 4, 2, 40, 15), 0),
     }[case]
     t_cpu = wl.make_tensors(w)
     t = {k: v.cuda() for k, v in t_cpu.items()}

@@ -66,6 +66,29 @@ def test_split_prompt_kv_head_dim_64(B):
     pu.assert_parity(got, pu.run_oracle(w, t))
 
 
+PADDED = [
+    _wl("d96", [300, 129], [[130, 257], [64]], 8, 2, 96, 31),        # 96 of a 128-wide tile
+    _wl("d80-gqa4", [513], [[200, 1, 129]], 8, 2, 80, 32),
+    _wl("d32", [260], [[140, 70]], 4, 4, 32, 33),                      # half of a 64-wide tile
+    _wl("d8", [130], [[65]], 2, 1, 8, 34),
+    _wl("d120", [200], [[100] * 3], 6, 3, 120, 35),
+]
+
+
+@pytest.mark.parametrize("w", PADDED, ids=[w.name for w in PADDED])
+@pytest.mark.parametrize("mode", ["plain", "sharded", "handoff"])
+def test_head_dims_below_the_tile_width(B, w, mode):
+    """Head dimensions that are not 64 or 128 run on the next wider tile: the tensor maps fill the missing columns with
+    zeros and the epilogues leave them out.  Guarded outputs: nothing may be written beyond a row's d columns (the rows
+    are contiguous, so a stray column would land in the next head's row and break parity there)."""
+    t = wl.make_tensors(w)
+    got, plan = pu.run_gpu(B, w, t, kv_splits=3 if mode == "sharded" else 0, handoff_limit=(1 << 40) if mode == "handoff" else 0)
+    if mode == "sharded":
+        assert plan.metadata(B.TBL_GROUP_SPLITS).max() > 1
+    wide = {k: {"rel_l2": 1.2e-2} for k in ("o_p", "o_r", *pu.GRADS)} if w.head_dim == 8 else None   # 8 numbers per row: no averaging
+    pu.assert_parity(got, pu.run_oracle(w, t), exceptions=wide)
+
+
 @pytest.mark.parametrize("gain", [4.0, 16.0])
 def test_large_norm_inputs_take_the_tracked_maximum_path(B, gain):
     """The forward kernel leaves the softmax reference at the first tile's row maximum when |q| max|k| scale

@@ -33,8 +33,12 @@ def test_descriptor_validation(binding):
         B.Plan([16], [[4]], 3, 2, 64, device=None, n_lanes=4)
     assert e.value.code == -2                    # h_q % h_kv
     with pytest.raises(B.AugtreeError) as e:
-        B.Plan([16], [[4]], 4, 2, 96, device=None, n_lanes=4)
-    assert e.value.code == -2                    # head_dim
+        B.Plan([16], [[4]], 4, 2, 100, device=None, n_lanes=4)
+    assert e.value.code == -2                    # head_dim not a multiple of 8
+    with pytest.raises(B.AugtreeError) as e:
+        B.Plan([16], [[4]], 4, 2, 136, device=None, n_lanes=4)
+    assert e.value.code == -2                    # head_dim above the tile width
+    assert B.Plan([16], [[4]], 4, 2, 96, device=None, n_lanes=4).head_dim == 96
     with pytest.raises(B.AugtreeError) as e:
         B.Plan([0], [[4]], 4, 2, 64, device=None, n_lanes=4)
     assert e.value.code == -1                    # empty prompt
