@@ -335,6 +335,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-configs", action="store_true", help="skip the brief runs of the other four configurations")
+    ap.add_argument("--scale-down", type=int, default=1,
+                    help="divide every length of the configuration by this (small cases of the same kernels for ncu captures; "
+                         "the workload's name in `config` carries the divisor)")
+    ap.add_argument("--bwd-handoff", action="store_true",
+                    help="backward calls take the dS hand-off path (5 GEMMs per tile pair, 32 KB of scratch per pair and head)")
     ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
                     help="weak (default): every rank runs its own groups; strong: one workload partitioned over the ranks")
     args = ap.parse_args()
@@ -343,7 +348,9 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    w = wl.config(args.config)
+    w = wl.config(args.config, args.scale_down)
+    if args.scale_down != 1:
+        w.name = f"{w.name}/{args.scale_down}"
 
     if args.impl == "reference":
         if rank == 0:
@@ -378,7 +385,9 @@ def main():
     plan = B.Plan(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, device=local_rank, flags=B.FLAG_ZERO_PROMPT_GRAD,
                   kv_splits=splits)
     plan_ms = (time.perf_counter() - t_plan) * 1e3  # pack and schedule on the host + table upload; not part of a step
-    out = B.alloc_outputs(plan)
+    out = B.alloc_outputs(plan, handoff_limit=(1 << 62) if args.bwd_handoff else 0)
+    handoff = out["ws"].numel() >= plan.ws_bwd_handoff_bytes
+    out_ws_bytes = out["ws"].numel()
 
     def step():
         B.run_forward_backward(plan, t_dev, out)
@@ -400,14 +409,15 @@ def main():
     # dominant kernel: the replay backward tile kernel
     names = ["prefill_fwd", "replay_fwd", "replay_bwd_dkdv", "prefill_bwd_dkdv", "replay_bwd_dq", "prefill_bwd_dq"]
     kfun = {"prefill_fwd": "fwd_kernel", "replay_fwd": "fwd_kernel", "replay_bwd_dkdv": "bwd_kernel", "prefill_bwd_dkdv": "bwd_kernel",
-            "replay_bwd_dq": "dq_kernel", "prefill_bwd_dq": "dq_kernel"}
+            "replay_bwd_dq": "dql_kernel" if handoff else "dq_kernel", "prefill_bwd_dq": "dql_kernel" if handoff else "dq_kernel"}
     per_kernel = {}
     for n, (tot, cnt) in zip(names, kt):
         if cnt:
             # tflops: the GEMM FLOPs the launch executes; tflops_algorithmic: its share of the 14 d per pair (the
             # query-side kernel's S and dP are recomputation: only its dQ GEMM, 2 d of its 6 d, is algorithmic)
             alg = fl[n] / 3 if n.endswith("_dq") else fl[n]
-            per_kernel[n] = {"ms": tot / cnt, "tflops": fl[n] / (tot / cnt * 1e-3) / 1e12,
+            executed = alg if handoff else fl[n]     # on the hand-off path the query-side launch is the dQ GEMM alone
+            per_kernel[n] = {"ms": tot / cnt, "tflops": executed / (tot / cnt * 1e-3) / 1e12,
                              "tflops_algorithmic": alg / (tot / cnt * 1e-3) / 1e12, "launches": cnt}
     dom = max(per_kernel, key=lambda n: per_kernel[n]["ms"])
     roofline = {"bound": "tensor", "kernel": f"{kfun[dom]} ({dom})", "achieved": per_kernel[dom]["tflops"],
@@ -461,7 +471,7 @@ def main():
 
     # ---- the other four configurations, briefly (3 timed steps each; `value` stays the default workload's)
     others = None
-    if rank == 0 and world == 1 and args.config == 2 and not args.no_configs:
+    if rank == 0 and world == 1 and args.config == 2 and args.scale_down == 1 and not args.no_configs:
         del out, t_dev
         torch.cuda.empty_cache()
         others = {}
@@ -484,6 +494,8 @@ def main():
             "pct_of_nominal_bf16_peak": 100 * value / world / NOMINAL_BF16_TFLOPS,
             "kernels": per_kernel, "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "flattened": flat, "cpu_baseline": cpu, "configs": others,
+            "bwd_path": "dS hand-off (5 GEMMs per tile pair)" if handoff else "recompute (7 GEMMs per tile pair)",
+            "bwd_scratch_bytes": int(out_ws_bytes),
         }
         print(json.dumps(line), flush=True)
     if dist is not None:
