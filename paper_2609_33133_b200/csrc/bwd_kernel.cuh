@@ -98,7 +98,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   const uint32_t bar_q_full = bars + 16, bar_q_empty = bars + 48;     // [NST <= 4] each
   const uint32_t bar_do_full = bars + 80, bar_do_empty = bars + 112;  // [NST <= 4] each
   const uint32_t bar_s_full = bars + 144, bar_p_ready = bars + 152, bar_dp_full = bars + 160, bar_ds_ready = bars + 168;
-  const uint32_t bar_acc_full = bars + 176, bar_acc_empty = bars + 184;
+  const uint32_t bar_acc_full = bars + 176, bar_acc_empty = bars + 184, bar_p_hi = bars + 208;
   volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_raw + SM::kOffBar + 192);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + SM::kOffBar + 200);
 
@@ -109,7 +109,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       mbar_init(bar_q_full + 8 * s, 1); mbar_init(bar_q_empty + 8 * s, 1);
       mbar_init(bar_do_full + 8 * s, 1); mbar_init(bar_do_empty + 8 * s, 1);
     }
-    mbar_init(bar_s_full, 1); mbar_init(bar_p_ready, 16); mbar_init(bar_dp_full, 1); mbar_init(bar_ds_ready, 16);
+    mbar_init(bar_s_full, 1); mbar_init(bar_p_ready, 16); mbar_init(bar_p_hi, 16); mbar_init(bar_dp_full, 1); mbar_init(bar_ds_ready, 16);
     mbar_init(bar_acc_full, 1); mbar_init(bar_acc_empty, 16);
     *abort_flag = 0;
     fence_barrier_init();
@@ -232,11 +232,18 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           }
           ok = need(have_p, bar_p_ready, T & 1, WAIT_BWD_PDS_FULL);
           if (!ok) break;
-          // (query columns 16k..16k+15: P^T sits at R0 columns 32 (k / 2) + 8 (k % 2), over its own thread's S^T)
-          mma_group<8>(elected,
-                       [&](int k) {
-                         mma_ts2(tDV, tR0 + 32 * (k >> 1) + 8 * (k & 1), dom_lo + kstep_mnmajor(k), IDESC_ACC, acc0 | (uint32_t)(k > 0));
-                       },
+          // (query columns 16k..16k+15: P^T sits at R0 columns 32 (k / 2) + 8 (k % 2), over its own thread's S^T.)
+          // Every element-wise warp hands over the first 16 of its 32 query columns (the even k steps) while it is
+          // still exponentiating the rest, so half of this GEMM runs under the second half of the P phase: the loop
+          // dV(T) -> S(T+1) -> P(T+1) -> dV(T+1) is what bounds a pair.
+          bool have_hi = false;
+          mma_group<4>(elected,
+                       [&](int k) { mma_ts2(tDV, tR0 + 32 * k, dom_lo + kstep_mnmajor(2 * k), IDESC_ACC, acc0 | (uint32_t)(k > 0)); },
+                       [&]() { have_hi = mbar_test(bar_p_hi, T & 1); });
+          ok = need(have_hi, bar_p_hi, T & 1, WAIT_BWD_PDS_FULL);
+          if (!ok) break;
+          mma_group<4>(elected,
+                       [&](int k) { mma_ts2(tDV, tR0 + 32 * k + 8, dom_lo + kstep_mnmajor(2 * k + 1), IDESC_ACC, 1u); },
                        [&]() { have_q = more && mbar_test(bar_q_full + 8 * st1, par1); });
           if (elected) tc_commit(bar_do_empty + 8 * st);
           // ---- S^T(T+1) = K Q^T -> R0 (free: dV(T) was issued and the tensor pipe runs in order)
@@ -290,31 +297,33 @@ bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       tmem_ld32(tR0 + lane_off + ch * 32, sv);
       tc_wait_ld();
       // packed fp32: one fma per pair for the scale-and-subtract (the table holds -lse*log2e), and the pairs
-      // that kBwdFmaMask names take their exp2 on the FMA pipe
+      // that kBwdFmaMask names take their exp2 on the FMA pipe.  Two halves of 16 query columns, each handed
+      // to the MMA warp as soon as it is in TMEM.
       const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
 #pragma unroll
-      for (int i = 0; i < 32; i += 4) {
-        const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + i);
-        const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(sv[i + 0]), __uint_as_float(sv[i + 1])), sc2, make_float2(l4.x, l4.y));
-        const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])), sc2, make_float2(l4.z, l4.w));
-        const float2 p0 = ((kBwdFmaMask >> (i / 2)) & 1) ? ex2_fma2(x0) : ex2_2(x0);
-        const float2 p1 = ((kBwdFmaMask >> (i / 2 + 1)) & 1) ? ex2_fma2(x1) : ex2_2(x1);
-        pr[i + 0] = p0.x; pr[i + 1] = p0.y; pr[i + 2] = p1.x; pr[i + 3] = p1.y;
-      }
-      if (!all_visible) {
+      for (int h = 0; h < 2; ++h) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (!key_valid || ch * 32 + i < lo) pr[i] = 0.f;
-      }
-      {
-        uint32_t pk[16];
+        for (int i = 16 * h; i < 16 * h + 16; i += 4) {
+          const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + i);
+          const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(sv[i + 0]), __uint_as_float(sv[i + 1])), sc2, make_float2(l4.x, l4.y));
+          const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])), sc2, make_float2(l4.z, l4.w));
+          const float2 p0 = ((kBwdFmaMask >> (i / 2)) & 1) ? ex2_fma2(x0) : ex2_2(x0);
+          const float2 p1 = ((kBwdFmaMask >> (i / 2 + 1)) & 1) ? ex2_fma2(x1) : ex2_2(x1);
+          pr[i + 0] = p0.x; pr[i + 1] = p0.y; pr[i + 2] = p1.x; pr[i + 3] = p1.y;
+        }
+        if (!all_visible) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(pr[2 * i], pr[2 * i + 1]);
-        tmem_st16(tR0 + lane_off + ch * 32, pk);
+          for (int i = 16 * h; i < 16 * h + 16; ++i)
+            if (!key_valid || ch * 32 + i < lo) pr[i] = 0.f;
+        }
+        uint32_t pk[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pk[i] = pack_bf16(pr[16 * h + 2 * i], pr[16 * h + 2 * i + 1]);
+        tmem_st8(tR0 + lane_off + ch * 32 + 8 * h, pk);
+        tc_wait_st();
+        tc_fence_before();
+        warp_arrive(h ? bar_p_hi : bar_p_ready);
       }
-      tc_wait_st();
-      tc_fence_before();
-      warp_arrive(bar_p_ready);
       return true;
     };
 
