@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libaugtree.so")
 SOURCES = ["augtree.cu", "plan.cpp", "planner.cpp"]
-HEADERS = ["ptx.cuh", "fwd_kernel.cuh", "bwd_kernel.cuh", "dq_kernel.cuh", "plan.h", os.path.join("..", "..", "include", "augtree.h")]
+HEADERS = ["ptx.cuh", "fwd_kernel.cuh", "bwd_kernel.cuh", "dq_kernel.cuh", "dql_kernel.cuh", "plan.h", os.path.join("..", "..", "include", "augtree.h")]
 
 
 def _stale() -> bool:
