@@ -155,3 +155,46 @@ def test_planner_solve_time_grows_mildly(B):
         times[blocks] = (time.perf_counter() - t0) / 20 * 1e3
     print("planner ms per tree:", {k: round(v, 3) for k, v in times.items()})
     assert max(times.values()) < 50.0
+
+
+def test_library_planner_above_the_exact_solver_cap(B):
+    """With more units than the exact AssignGrid solver takes, the library places each candidate largest-first; the
+    selection must then be Algorithm 1 over those placements: every candidate scored with Eq. 7-10 (the oracle's cost
+    functions) at the greedy placement (the oracle's restatement of the rule), the cheapest kept, first on ties."""
+    from oracle import packing
+    rng = np.random.default_rng(23)
+    for trial in range(25):
+        G = int(rng.integers(9, 30))
+        P = int(rng.choice([700, 4096, 20000, 65536]))
+        R = [int(rng.choice([64, 200, 513, 3000, 9000])) for _ in range(G)]
+        degrees = [2, 4, 8]
+        u = lambda lo, hi: float(rng.uniform(lo, hi))
+        prof = _prof(alpha_p=u(0, 0.1), beta_p=u(0, 0.01), lat_p0=u(0, 20), alpha_tmkv=u(0.5, 2), beta_tmkv=u(0, 0.01), lat_tmkv0=u(0, 20),
+                     lat_tmkv1=u(0, 2), alpha_mq=u(0.5, 2), beta_q=u(0, 0.005), red0=u(0, 10), red1=u(0, 0.005), lat_mq0=u(0, 20),
+                     lat_mq1=u(0, 5), alpha_ring=u(0.5, 2), beta_ring=u(0, 0.01), lat_ring0=u(0, 20), gamma_tmkv=u(0.8, 1.2), gamma_mq=u(0.8, 1.2))
+        if trial % 2:
+            prof.mem_prompt, prof.mem_resp, prof.mem_cap = 1.0, 1.0, float(P + sum(R) / 3)
+        w = [op.replay_tiles(P, r) for r in R]
+        best = None
+        for d, primitive, b, s in op.candidates(P, R, degrees, b_max=3):
+            if primitive == op.RING_CP:
+                if not op.ring_feasible(prof, P, R, d):
+                    continue
+                cand = (op.ring_cost(prof, P, R, 8, 2, d), d, primitive, 0, 1, None)
+            else:
+                cap = op.cell_token_cap(prof, primitive, P, d, s)
+                if cap is not None and cap < 0:
+                    continue
+                placed = packing.greedy_grid(w, R, b, s, cap)
+                if placed is None:
+                    continue
+                cand = (op.split_cost(prof, primitive, P, R, 8, 2, d, b, s, placed[2]), d, primitive, b, s, placed)
+            if best is None or cand[0] < best[0]:
+                best = cand
+        got = B.plan_tree(P, R, 8, 2, degrees, _as_dict(prof), b_max=3, exact_max_units=8)
+        assert best is not None
+        assert got["cost"] == pytest.approx(best[0], rel=1e-12), (trial, got, best[:5])
+        assert (got["degree"], got["primitive"], got["rounds"], got["lanes"]) == best[1:5], (trial, got, best[:5])
+        if best[2] != op.RING_CP:
+            assert not got["solved_exactly"]
+            assert (got["X"][0], got["X"][1]) == (best[5][0], best[5][1])       # the greedy rule is deterministic: same placement
