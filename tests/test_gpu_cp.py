@@ -27,6 +27,7 @@ CASES = {
     "two-groups": wl.Workload("moveq-a", [700, 300], [[300, 150, 420], [257]], 4, 2, 128, 81),
     "gqa7-d128": wl.Workload("moveq-b", [1100], [[130, 64, 200, 90, 333]], 14, 2, 128, 82),
     "d64": wl.Workload("moveq-c", [513, 260], [[129, 1], [300, 77]], 8, 2, 64, 83),
+    "d96": wl.Workload("moveq-d", [640], [[200, 130, 65]], 8, 2, 96, 85),     # head dimension padded to the 128-wide tile
 }
 
 

@@ -12,7 +12,7 @@ import torch.nn.functional as F
 
 pytestmark = pytest.mark.gpu
 
-HIDDEN, H_Q, H_KV, D, MLP, VOCAB, LAYERS = 256, 4, 2, 64, 512, 503, 2
+HIDDEN, H_Q, H_KV, MLP, VOCAB, LAYERS = 256, 4, 2, 512, 503, 2
 
 
 @pytest.fixture(scope="module")
@@ -24,7 +24,7 @@ def mods():
 
 
 class TinyLM(torch.nn.Module):
-    def __init__(self, L):
+    def __init__(self, L, D):
         super().__init__()
         self.emb = torch.nn.Parameter(torch.randn(VOCAB, HIDDEN) * 0.5)
         self.layers = torch.nn.ModuleList([L.TreeDecoderLayer(HIDDEN, H_Q, H_KV, D, MLP) for _ in range(LAYERS)])
@@ -67,7 +67,8 @@ def flat_loss(L, model, prompt_len, branch_len, prompt_tok, resp_tok):
     return total
 
 
-def test_tree_and_flattened_training_agree(mods):
+@pytest.mark.parametrize("D", [64, 96])
+def test_tree_and_flattened_training_agree(mods, D):
     B, L = mods
     torch.manual_seed(11)
     prompt_len, branch_len = [300, 129], [[130, 64, 257, 1], [200, 33]]
@@ -75,7 +76,7 @@ def test_tree_and_flattened_training_agree(mods):
     g = torch.Generator().manual_seed(3)
     prompt_tok = torch.randint(0, VOCAB, (sum(prompt_len),), generator=g).cuda()
     resp_tok = torch.randint(0, VOCAB, (sum(sum(b) for b in branch_len),), generator=g).cuda()
-    tree_model = TinyLM(L).cuda()
+    tree_model = TinyLM(L, D).cuda()
     flat_model = copy.deepcopy(tree_model)
 
     # ---- one step: loss and the gradient of every weight
