@@ -5,9 +5,9 @@ Input: the raw-page CSV of an ncu capture of bench.py (tile kernels only, whole 
 
     CMD="python bench.py --steps 2 --warmup 3 --no-flattened --no-cpu-baseline --no-e2e --no-configs"
     $CMD && ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --clock-control none \\
-        -k regex:"fwd_kernel|bwd_kernel|dq_kernel" -s 6 -c 6 -f -o gpurun_out/prof_dram $CMD
-    ncu -i gpurun_out/prof_dram.ncu-rep --page raw --csv > gpurun_out/prof_dram.csv
-    python bench_ncu_bytes.py gpurun_out/prof_dram.csv cfg2-7b-layer "<the ncu command>"
+        -k regex:"fwd_kernel|bwd_kernel|dq_kernel" -s 6 -c 6 -f -o prof_dram $CMD
+    ncu -i prof_dram.ncu-rep --page raw --csv > prof_dram.csv
+    python bench_ncu_bytes.py prof_dram.csv cfg2-7b-layer "<the ncu command>"
 
 One step launches, in order: fwd_kernel (prefill), fwd_kernel (replay), bwd_kernel (replay), dq_kernel (replay),
 bwd_kernel (prefill), dq_kernel (prefill); the capture must start at a step boundary.
