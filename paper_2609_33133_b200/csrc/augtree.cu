@@ -186,7 +186,9 @@ template <int D>
 int launch_bwd(const augtree_plan *pl, const Sched &s, const BwdArgs &a, void *ws, size_t ws_bytes, cudaStream_t st) {
   if (a.q_tok == 0) return AUGTREE_OK;
   float *stats = static_cast<float *>(ws);
-  const bool handoff = ws_bytes >= pl->ws_bwd_handoff && s.n_items() > 0 && a.dq_sched->n_items() > 0;
+  // (the hand-off tiles are written with 32-byte stores: the scratch must be aligned to that, else the recomputing path)
+  const bool handoff = ws_bytes >= pl->ws_bwd_handoff && s.n_items() > 0 && a.dq_sched->n_items() > 0 &&
+                       (reinterpret_cast<uintptr_t>(ws) & 31u) == 0;
   __nv_bfloat16 *ds = handoff ? reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(ws) + pl->ws_bwd) : nullptr;
   {
     const dim3 grid((unsigned)a.n_tiles, (unsigned)pl->h_q);

@@ -73,3 +73,29 @@ def test_partial_state_backward_takes_the_handoff_too(B):
         assert torch.equal(dk_a, dk_b) and torch.equal(dv_a, dv_b)
         err = (dq_a - dq_b).abs().max().item()
         assert err <= 1e-3 * max(1.0, dq_a.abs().max().item()), err   # same bf16 dS, fp32 sums in the same order
+
+
+def test_workspace_aligned_to_16_bytes_only_takes_the_recomputing_path(B):
+    """The hand-off tiles are written with 32-byte stores; a scratch block that is large enough but only 16-byte aligned
+    must not take that path: its dQ is then bit for bit the recomputing kernel's."""
+    w = wl.Workload("align", [400], [[150, 260]], 4, 2, 128, seed=9)
+    t = {k: v.cuda() for k, v in wl.make_tensors(w, device="cpu").items()}
+    plan = B.Plan(w.prompt_len, w.branch_len, w.h_q, w.h_kv, w.head_dim, device=0)
+    out = B.alloc_outputs(plan, handoff_limit=0)
+    B.run_forward_backward(plan, t, out)
+    torch.cuda.synchronize()
+    want = {k: out[k].clone() for k in ("dq_r", "dk_r", "dv_r", "dk_p", "dv_p")}
+    big = torch.empty(plan.ws_bwd_handoff_bytes + 64, device="cuda", dtype=torch.uint8)
+    off = (-big.data_ptr()) % 32 + 16                     # 16 modulo 32
+    ws = big[off:off + plan.ws_bwd_handoff_bytes]
+    assert ws.data_ptr() % 32 == 16 and ws.numel() >= plan.ws_bwd_handoff_bytes
+    out["dk_p"].zero_(); out["dv_p"].zero_()
+    for k in ("dq_r", "dk_r", "dv_r"):
+        out[k].fill_(float("nan"))
+    plan.replay_bwd(t["q_r"], t["k_r"], t["v_r"], t["k_p"], t["v_p"], out["o_r"], out["lse_r"], t["do_r"],
+                    out["dq_r"], out["dk_r"], out["dv_r"], out["dk_p"], out["dv_p"], ws)
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0)
+    # dk_p / dv_p of the reference run also hold the prefill call's share: compare the replay outputs only
+    for k in ("dq_r", "dk_r", "dv_r"):
+        assert torch.equal(out[k], want[k]), k
