@@ -253,7 +253,8 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
   p->ws_bwd = al(hq * ntile * 2 * kTileQ * 4);
   // with this much, the key-side kernel also stores dS (bf16, one 128 x 128 tile per pair and head) for the query side
   const int64_t ds_slots = std::max(p->ds_slots_replay, p->ds_slots_prefill);
-  p->ws_bwd_handoff = ds_slots > 0x3fffffff ? ~(size_t)0 : p->ws_bwd + al((size_t)ds_slots * hq * (size_t)(kTileQ * kTileKV * 2));
+  // (slot indices are 32-bit tensor-map coordinates)
+  p->ws_bwd_handoff = ds_slots * (int64_t)p->h_q > 0x7fffffff ? ~(size_t)0 : p->ws_bwd + al((size_t)ds_slots * hq * (size_t)(kTileQ * kTileKV * 2));
   (void)tmax; (void)dd;
   return AUGTREE_OK;
 }
