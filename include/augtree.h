@@ -287,8 +287,8 @@ int augtree_last_device_status(const augtree_plan_t *plan, int *status, int *det
  * that holds one shard of the keys computes, for every response query it is given, the PARTIAL online-softmax
  * state over that shard; the states of a query are merged afterwards (the (+) of Sec. 3.3), on whichever rank
  * owns the query; in the backward pass every shard owner computes its shard's dK, dV and its contribution to dQ
- * from the merged LSE, and the dQ contributions are summed on the way back ("its custom autograd operator applies
- * the reverse communication", Sec. 3.3).  These three calls are the per-rank compute steps; moving queries,
+ * from the merged LSE, and the dQ contributions are summed on the way back (in the backward pass of MoveQ the
+ * exchange of the forward pass runs in reverse, Sec. 3.3).  These three calls are the per-rank compute steps; moving queries,
  * states and gradients between ranks is the caller's (NCCL or peer copies, no multicast loads).  state_o,
  * state_lse and dq_part are written with plain global stores from the tile kernels' epilogues, so they may be
  * peer-mapped memory of the rank that will merge them: the exchange then happens as the tiles finish.  Inputs

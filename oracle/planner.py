@@ -68,7 +68,7 @@ def f_ring(d):
 
 def replay_tiles(P, R):
     """Valid Q-KV tiles of one response path in replay: every response query tile against every prompt tile, plus the
-    causal triangle of its own tiles (unit weight w_k: 'query length, valid Q-KV tile count', Sec. 3.4)."""
+    causal triangle of its own tiles (the weight w_k of a replay unit in Sec. 3.4 is its count of valid tiles)."""
     nq = cdiv(R, TILE)
     return nq * cdiv(P, TILE) + nq * (nq + 1) // 2
 
@@ -97,8 +97,8 @@ def cell_token_cap(prof: Profile, primitive, P, d, s):
 
 
 def cell_tokens_proxy(R, b, s):
-    """Response tokens of the fullest cell, estimated without looking at the placement: 'the implementation uses
-    L_R^max = max_i |R_i| as a conservative replay-length proxy' (Sec. 3.4), here for ceil(G / (b s)) paths per cell
+    """Response tokens of the fullest cell, estimated without looking at the placement: Sec. 3.4 lets the longest
+    response length max_i |R_i| stand in, conservatively, for the replay length; here for ceil(G / (b s)) paths per cell
     [reading].  The traffic terms then depend on the candidate alone and the placement enters through W only."""
     return cdiv(len(R), b * s) * max(R)
 

@@ -8,7 +8,7 @@ rank computes every query's partial softmax state over its prompt-KV shard (plus
 branch's own causal prefix), and the n states of a query are merged on its owner.  Backward: the merged output,
 its LSE and the seed dO are made known to every rank; each rank computes its shard's dK_P / dV_P (complete: the
 many-to-one sum of Eq. 2 is local to the shard's owner), dK_R / dV_R of the branches it owns, and its contribution
-to every dQ; the dQ contributions are summed on the way back to the queries' owners (the reverse communication).
+to every dQ; the dQ contributions are summed on the way back to the queries' owners (the forward exchange run in reverse).
 
 The per-rank compute steps are calls into the library (`CudaBackend`: augtree_replay_fwd_state, augtree_merge_states,
 augtree_replay_bwd_state); what remains here is bookkeeping and the exchange steps.  `moveq_emulate` runs all ranks
@@ -218,7 +218,7 @@ def moveq_rank(dist, backend, w, rank: int, world: int, local: Dict[str, torch.T
     do_all = everywhere(local["do_r"])
     dq_part, dk_r, dv_r, dkp, dvp = bwd_compute(backend, w, lay, q_all, local["k_r"], local["v_r"], local["k_p"], local["v_p"],
                                                 o_all, lse_all, do_all)
-    dist.all_reduce(dq_part, op=dist.ReduceOp.SUM)         # the reverse communication
+    dist.all_reduce(dq_part, op=dist.ReduceOp.SUM)         # the forward exchange in reverse
     mine = torch.zeros(q_all.shape[0], dtype=torch.bool, device=q_all.device)
     if lay.owned:
         mine[torch.as_tensor(_rows(lay, lay.owned), device=q_all.device)] = True

@@ -1,8 +1,8 @@
 """One decoder layer and the language-model loss on a prompt-sharing tree (integration around the attention path).
 
-What the method changes in a model is its self-attention operator and nothing else: "these are the only
-model-operator changes; losses, gradient synchronization, and optimizer steps remain those of the base trainer"
-(Sec. 4, attention dispatch).  This module is that seam written out for a standard pre-norm decoder layer:
+What the method changes in a model is its self-attention operator and nothing else: loss, gradient synchronisation
+and optimizer stay the base trainer's (Sec. 4, attention dispatch).  This module is that seam written out for a
+standard pre-norm decoder layer:
 
 * the prompt of a group is embedded and pushed through the layer ONCE, its responses once each, never the G flattened
   copies (Sec. 3.2, prefill once / replay);
@@ -11,9 +11,8 @@ model-operator changes; losses, gradient synchronization, and optimizer steps re
 * attention: `autograd.tree_attention` (the C-ABI path; everything else here is plain torch: library GEMMs,
   element-wise ops);
 * loss: token-level cross-entropy on the response tokens.  The first token of every response is scored from the
-  LAST PROMPT hidden state of its group ("scored by applying the language-model head to the final prompt hidden
-  state from the prefill pass, and its loss backpropagates through that state into the prompt graph", Sec. 3.2):
-  that state therefore carries one target per branch.
+  LAST PROMPT hidden state of its group, and that loss flows back through the prompt's own graph (Sec. 3.2, response
+  replay): that state therefore carries one target per branch.
 
 Nothing here is on the measured hot path; tests compare loss and weight gradients with the flattened execution.
 """

@@ -128,7 +128,7 @@ TENSOR_NAMES = ("q_p", "k_p", "v_p", "do_p", "q_r", "k_r", "v_r", "do_r")
 
 # --------------------------------------------------------------------------- #
 # Sharding over GPUs without any exchange step.  Replay trees are independent of
-# each other (the paper's CP groups "run different trees", Sec. 3.5) and, inside
+# each other (data-parallel replicas work on different trees, Sec. 3.5) and, inside
 # attention, so are KV heads: a KV head with the query heads that read it can live
 # on one GPU, and the many-to-one prompt-KV gradient of Eq. 2 stays local to it.
 # So the units are whole groups when there are at least as many groups as ranks,

@@ -2,8 +2,8 @@
 prompt-sharing tree (prompt once, responses replayed, first response token scored from the last prompt state) against
 the same model on the flattened sequences (every branch as its own prompt + response sequence, plain causal
 attention in torch).  Loss and weight gradients must agree, and so must the loss trajectory over a few optimizer
-steps: the check the paper reports for its engine ("matching loss trajectories ... under identical replay inputs",
-Sec. 5, correctness)."""
+steps: the check the paper reports for its engine (equal loss trajectories on identical replay inputs, Sec. 5,
+correctness)."""
 import copy
 
 import pytest
