@@ -30,33 +30,57 @@ namespace augtree {
 
 static inline int cdiv(int a, int b) { return (a + b - 1) / b; }
 
-static void assign_lanes(Sched &s, int weight_field, int n_lanes) {
+// Returns false when the sizes do not fit the packed heap keys (lane index in 20 bits, lane load above them).
+static bool assign_lanes(Sched &s, int weight_field, int n_lanes) {
   const int n = s.n_items();
-  std::vector<int32_t> ids(n);
-  std::iota(ids.begin(), ids.end(), 0);
   const int32_t *it = s.items.data();
   const int ni = s.item_ints;
-  std::stable_sort(ids.begin(), ids.end(), [&](int32_t a, int32_t b) {
-    return it[(size_t)a * ni + weight_field] > it[(size_t)b * ni + weight_field];
-  });
-  typedef std::pair<int64_t, int32_t> LL;  // (load, lane): smallest load first, then lowest lane
-  std::priority_queue<LL, std::vector<LL>, std::greater<LL>> heap;
-  for (int l = 0; l < n_lanes; ++l) heap.push(LL(0, l));
-  std::vector<std::vector<int32_t>> per_lane(n_lanes);
+  // ids by weight descending, id ascending inside a weight: a counting sort (weights are tile counts, small integers)
+  int32_t wmax = 0;
+  int64_t wsum = 0;
+  for (int i = 0; i < n; ++i) { wmax = std::max(wmax, it[(size_t)i * ni + weight_field]); wsum += it[(size_t)i * ni + weight_field]; }
+  if (n_lanes > (1 << 20) || wsum >= ((int64_t)1 << 43)) return false;
+  std::vector<int32_t> ids(n);
+  if ((int64_t)wmax <= 4 * (int64_t)n + 1024) {
+    std::vector<int32_t> start((size_t)wmax + 2, 0);
+    for (int i = 0; i < n; ++i) ++start[(size_t)(wmax - it[(size_t)i * ni + weight_field]) + 1];
+    for (size_t b = 1; b < start.size(); ++b) start[b] += start[b - 1];
+    for (int i = 0; i < n; ++i) ids[start[(size_t)(wmax - it[(size_t)i * ni + weight_field])]++] = i;
+  } else {
+    std::iota(ids.begin(), ids.end(), 0);
+    std::stable_sort(ids.begin(), ids.end(), [&](int32_t a, int32_t b) {
+      return it[(size_t)a * ni + weight_field] > it[(size_t)b * ni + weight_field];
+    });
+  }
+  // largest first, each to the lane with the smallest (load, lane index): a binary min-heap of keys
+  // load * 2^20 + lane whose top is replaced in place (one sift-down per item)
+  std::vector<uint64_t> heap(n_lanes);
+  std::vector<int32_t> lane_of(n), count(n_lanes + 1, 0);
+  for (int l = 0; l < n_lanes; ++l) heap[l] = (uint64_t)l;   // all loads 0: ascending lane index is a valid heap
+  uint64_t *hp = heap.data();
   for (int32_t id : ids) {
-    LL top = heap.top();
-    heap.pop();
-    per_lane[top.second].push_back(id);
-    heap.push(LL(top.first + it[(size_t)id * ni + weight_field], top.second));
+    const int32_t lane = (int32_t)(hp[0] & 0xfffffu);
+    lane_of[id] = lane;
+    ++count[lane + 1];
+    const uint64_t key = hp[0] + ((uint64_t)it[(size_t)id * ni + weight_field] << 20);
+    int i = 0;
+    while (true) {
+      int c = 2 * i + 1;
+      if (c >= n_lanes) break;
+      if (c + 1 < n_lanes && hp[c + 1] < hp[c]) ++c;
+      if (hp[c] >= key) break;
+      hp[i] = hp[c];
+      i = c;
+    }
+    hp[i] = key;
   }
+  // inside a lane items run in ascending id: one pass over the ids in order
   s.lane_ptr.assign(n_lanes + 1, 0);
-  s.order.clear();
-  s.order.reserve(n);
-  for (int l = 0; l < n_lanes; ++l) {
-    std::sort(per_lane[l].begin(), per_lane[l].end());
-    s.order.insert(s.order.end(), per_lane[l].begin(), per_lane[l].end());
-    s.lane_ptr[l + 1] = (int32_t)s.order.size();
-  }
+  for (int l = 0; l < n_lanes; ++l) s.lane_ptr[l + 1] = s.lane_ptr[l] + count[l + 1];
+  s.order.assign(n, 0);
+  std::vector<int32_t> fill(s.lane_ptr.begin(), s.lane_ptr.end() - 1);
+  for (int i = 0; i < n; ++i) s.order[fill[lane_of[i]]++] = i;
+  return true;
 }
 
 int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
@@ -151,6 +175,25 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
   pf.item_ints = rf.item_ints = rq.item_ints = pq.item_ints = AUGTREE_FWD_ITEM_INTS;
   rb.item_ints = pb.item_ints = AUGTREE_BWD_ITEM_INTS;
   pf.items.clear(); rf.items.clear(); rb.items.clear(); pb.items.clear(); rq.items.clear(); pq.items.clear();
+  {  // item counts, so that the tables below grow without reallocation
+    size_t n_pf = 0, n_rf = 0, n_rb = 0, n_pb = 0, n_rq = 0, n_pq = 0;
+    for (int g = 0; g < ng; ++g) {
+      const int P = p->prompt_len[g];
+      n_pf += (size_t)cdiv(P, kTileQF) * p->h_q;
+      n_pq += (size_t)cdiv(P, kTileQ) * p->h_q;
+      n_pb += (size_t)cdiv(P, kTileKV) * p->h_kv;
+      if (p->cu_b[g + 1] > p->cu_b[g]) n_rb += (size_t)cdiv(P, kTileKV) * p->h_kv;
+      for (int b = p->cu_b[g]; b < p->cu_b[g + 1]; ++b) {
+        const int R = p->branch_len[b];
+        n_rq += (size_t)cdiv(R, kTileQ) * p->h_q;
+        n_rf += (size_t)cdiv(R, kTileQF) * p->h_q * p->group_splits[g];
+        n_rb += (size_t)cdiv(R, kTileKV) * p->h_kv;
+      }
+    }
+    pf.items.reserve(n_pf * AUGTREE_FWD_ITEM_INTS); rf.items.reserve(n_rf * AUGTREE_FWD_ITEM_INTS);
+    rq.items.reserve(n_rq * AUGTREE_FWD_ITEM_INTS); pq.items.reserve(n_pq * AUGTREE_FWD_ITEM_INTS);
+    rb.items.reserve(n_rb * AUGTREE_BWD_ITEM_INTS); pb.items.reserve(n_pb * AUGTREE_BWD_ITEM_INTS);
+  }
 
   for (int g = 0; g < ng; ++g) {
     const int P = p->prompt_len[g], p0 = p->cu_p[g];
@@ -232,12 +275,9 @@ int build_plan_host(const augtree_desc_t *d, augtree_plan *p) {
     }
   }
   if (p->n_lanes > 0) {
-    assign_lanes(pf, 10, p->n_lanes);
-    assign_lanes(rf, 10, p->n_lanes);
-    assign_lanes(rb, 7, p->n_lanes);
-    assign_lanes(pb, 7, p->n_lanes);
-    assign_lanes(rq, 10, p->n_lanes);
-    assign_lanes(pq, 10, p->n_lanes);
+    if (!assign_lanes(pf, 10, p->n_lanes) || !assign_lanes(rf, 10, p->n_lanes) || !assign_lanes(rb, 7, p->n_lanes) ||
+        !assign_lanes(pb, 7, p->n_lanes) || !assign_lanes(rq, 10, p->n_lanes) || !assign_lanes(pq, 10, p->n_lanes))
+      return AUGTREE_ERR_UNSUPPORTED;
   }
 
   // scratch sizes (bytes, each region 256-byte aligned)
