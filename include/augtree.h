@@ -302,7 +302,9 @@ int augtree_last_device_status(const augtree_plan_t *plan, int *status, int *det
  *   over the keys {the plan's prompt} and, if include_own != 0, the query's own causal response prefix (k_r, v_r).
  *   The state is kept as (normalised O, LSE): the same information as (m, l, O_acc).
  * augtree_merge_states: merges n_states <= 16 such states (HOST arrays of DEVICE pointers) into o_r (bf16) and
- *   lse_r; a state whose LSE is -inf (no key seen) has weight zero.
+ *   lse_r; a state whose LSE is -inf (no key seen) has weight zero.  The states are read with plain global loads,
+ *   once each, so the pointers may also be peer-mapped memory of the ranks that computed them: the gather of
+ *   the states and their merge are then one kernel.
  * augtree_replay_bwd_state: with the MERGED o_r, lse_r and the seed do_r: dkp_acc, dvp_acc += gradients of the
  *   plan's prompt keys over all given queries (complete for this shard: Eq. 2's sum is local to the shard's owner);
  *   dq_part [sumR,H_q,d] fp32 = this shard's contribution to dQ (written, not added); with include_own != 0 also
