@@ -215,3 +215,14 @@ def test_handoff_scratch_counts_every_visible_tile_pair(binding):
         assert extra == max(replay, prefill) * hq * 128 * 128 * 2, (pl, bl)
         assert plan.workspace_bytes(0) == max(plan.ws_fwd_bytes, plan.ws_bwd_bytes, 256)
         assert plan.workspace_bytes(1 << 50) >= plan.ws_bwd_handoff_bytes
+
+
+def test_handoff_is_switched_off_when_a_slot_index_would_overflow(binding):
+    """Slot indices are 32-bit tensor-map coordinates: a plan with more than 2^31 (tile pair, head) slots reports
+    SIZE_MAX, so that no scratch size can select the hand-off path."""
+    B = binding
+    plan = B.Plan([1_200_000], [[]], 64, 8, 128, device=None, n_lanes=148)
+    tiles = -(-1_200_000 // 128)
+    assert tiles * (tiles + 1) // 2 * 64 > 2 ** 31
+    assert plan.ws_bwd_handoff_bytes == 2 ** 64 - 1
+    assert plan.workspace_bytes(2 ** 62) == max(plan.ws_fwd_bytes, plan.ws_bwd_bytes, 256)
