@@ -158,7 +158,9 @@ int augtree_plan_workspace_bytes(const augtree_plan_t *plan, size_t *fwd_bytes, 
  * given ws_bytes >= *bytes instead has the key-side kernel store dS (bf16, 32 KB per pair and query head:
  * *bytes = bwd_bytes + that, the larger of the two backward calls) and the query-side kernel compute
  * dQ = sum dS K from it: five GEMMs, at the price of writing and reading the scratch once.  Both paths give
- * dK, dV bit for bit the same and dQ from the same bf16 dS values summed in the same order.  *bytes is
+ * dK, dV bit for bit the same.  dQ then comes from the very dS values that went into dK instead of the query-side
+ * kernel's own recomputation of them (whose bf16 rounding of dS falls differently on a few per cent of the
+ * elements): the two paths' dQ agree to one bf16 step.  *bytes is
  * SIZE_MAX for a plan too large to index; the choice is the caller's, per call, through ws_bytes.  The path also
  * needs ws aligned to 32 bytes (the tiles are written with 32-byte stores); a less aligned ws takes the recomputing
  * path whatever its size.
