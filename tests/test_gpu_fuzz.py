@@ -49,9 +49,9 @@ SEEN = {
 }
 
 
-def _check(B, w, splits, lanes, flags):
+def _check(B, w, splits, lanes, flags, handoff_limit=None):
     t = wl.make_tensors(w)
-    got, _ = pu.run_gpu(B, w, t, kv_splits=splits, n_lanes=lanes, flags=flags)
+    got, _ = pu.run_gpu(B, w, t, kv_splits=splits, n_lanes=lanes, flags=flags, handoff_limit=handoff_limit)
     ref = pu.run_oracle(w, t)
     n_small = 2 * w.head_dim * w.h_q
     # a tensor of one or two rows: its relative-L2 figure is a couple of bf16 roundings, not a statistic
@@ -81,3 +81,17 @@ def test_random_small_workloads(B, case):
     if w.total_response == 0 and splits:
         splits = 0
     _check(B, w, splits, lanes, B.FLAG_ZERO_PROMPT_GRAD if case % 2 else 0)
+
+
+N_PADDED = 24
+
+
+@pytest.mark.parametrize("case", range(N_PADDED))
+def test_random_small_workloads_other_head_dims_and_handoff(B, case):
+    """The same sweep recipe (its own seeds) over head dimensions that are padded to the 64- or 128-column tile, on
+    the recomputing backward path (even cases) and on the dS hand-off path (odd cases)."""
+    w, splits, lanes = _random_case(1000 + case)
+    w.head_dim = int(np.random.default_rng(77 + case).choice([8, 16, 40, 56, 72, 80, 96, 104, 120]))
+    if w.total_response == 0 and splits:
+        splits = 0
+    _check(B, w, splits, lanes, B.FLAG_ZERO_PROMPT_GRAD if case % 3 else 0, handoff_limit=(1 << 40) if case % 2 else 0)
