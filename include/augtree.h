@@ -231,7 +231,9 @@ int augtree_replay_bwd(const augtree_plan_t *plan, const void *q_r, const void *
  * the seed do_p.  Its dK/dV are ADDED to dkp_acc/dvp_acc, which after this
  * call hold the final prompt-KV gradients (replay seeds + prefill graph,
  * Sec. 3.2); call it after augtree_replay_bwd on the same stream.  dq_p is
- * written; dk_p/dv_p (bf16 copies of the final accumulators) may be NULL.
+ * written; dk_p/dv_p (bf16 copies of the final accumulators) may be NULL,
+ * and then the two backward calls may come in either order: each adds its
+ * terms of the same sum to the fp32 accumulators.
  */
 int augtree_prefill_bwd(const augtree_plan_t *plan, const void *q_p, const void *k_p, const void *v_p,
                         const void *o_p, const float *lse_p, const void *do_p,

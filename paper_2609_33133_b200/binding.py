@@ -153,6 +153,7 @@ class Plan:
         self.prompt_len = [int(x) for x in prompt_len]
         self.branch_len = [[int(x) for x in b] for b in branch_len]
         self.h_q, self.h_kv, self.head_dim = h_q, h_kv, head_dim
+        self.softmax_scale, self.flags, self.n_lanes, self.kv_splits = softmax_scale, flags, n_lanes, kv_splits
         self.total_p = sum(self.prompt_len)
         self.total_r = sum(sum(b) for b in self.branch_len)
         n = len(self.prompt_len)
@@ -284,22 +285,61 @@ def run_forward_backward(plan: Plan, t, out):
 class HostStep:
     """The whole hot path for callers whose tensors live in (pinned) host memory: every input is copied to the device
     and every result back, with the copies overlapped with the kernels as far as the data flow allows.  Three streams:
-    one for the host->device copies in the order the calls need them (prompt inputs, response inputs, dO_R, dO_P), the
-    caller's current stream for the four entry points (each waits only for its own inputs), one for the device->host
-    copies (each result leaves as soon as its call has finished).  The caller's stream has joined both copy streams
-    when `run` returns (asynchronously, like the entry points).  Copies and waits only: no arithmetic here."""
+    one for the host->device copies in the order the calls need them, the caller's current stream for the entry points
+    (each waits only for its own inputs), one for the device->host copies (each result leaves as soon as its call has
+    finished).  The caller's stream has joined both copy streams when `run` returns (asynchronously, like the entry
+    points).  Copies, waits and slicing only: no arithmetic here.
+
+    chunks = 1: the four calls of the plan, inputs in the order (prompt inputs, response inputs, dO_R, dO_P).
+    chunks = K > 1: the response branches are cut, in packed order, into K runs of about equal length, each with a plan
+    of its own over the same prompts, and the replay calls run run by run: forward and backward of a run start as soon as
+    ITS slices have arrived, and its results leave while the next run computes.  The prompt-KV gradient accumulators take
+    one addition per run (Eq. 2's sum, associated differently from the single call: the same values to fp32 rounding);
+    everything else is bit for bit the single call's.  The prefill backward runs BEFORE the replay runs here (its share
+    of the accumulators is a term of the same sum, and no bf16 copy of them is asked for), so dQ_P leaves early."""
 
     IN_ORDER = (("q_p", "k_p", "v_p"), ("q_r", "k_r", "v_r"), ("do_r",), ("do_p",))
     OUT_ORDER = (("o_p", "lse_p"), ("o_r", "lse_r"), ("dq_r", "dk_r", "dv_r"), ("dq_p", "dk_p", "dv_p"))
 
-    def __init__(self, plan: Plan, dev_in, dev_out):
+    def __init__(self, plan: Plan, dev_in, dev_out, chunks=1):
         self.plan, self.t, self.out = plan, dev_in, dev_out
         self.s_in, self.s_out = torch.cuda.Stream(), torch.cuda.Stream()
         self.ev_in = [torch.cuda.Event() for _ in self.IN_ORDER]
         self.ev_done = [torch.cuda.Event() for _ in self.OUT_ORDER]
         self.ev_start, self.ev_in_end, self.ev_out_end = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
+        self.runs = self._make_runs(chunks) if chunks > 1 and plan.total_r > 0 else []
+
+    def _make_runs(self, chunks):
+        """Cut the packed branches into runs; per run: its plan, the row ranges of its responses and of its groups' prompts."""
+        plan = self.plan
+        branches = [(g, r) for g, rs in enumerate(plan.branch_len) for r in rs]
+        chunks = min(chunks, len(branches))
+        target, runs, b0, r0, acc = plan.total_r / chunks, [], 0, 0, 0
+        cu_p = [0]
+        for P in plan.prompt_len:
+            cu_p.append(cu_p[-1] + P)
+        for b, (g, r) in enumerate(branches):
+            acc += r
+            if acc >= target * (len(runs) + 1) - 1e-9 or b == len(branches) - 1:
+                g0, g1 = branches[b0][0], g
+                bl = [[] for _ in range(g0, g1 + 1)]
+                for gg, rr in branches[b0:b + 1]:
+                    bl[gg - g0].append(rr)
+                sub = Plan(plan.prompt_len[g0:g1 + 1], bl, plan.h_q, plan.h_kv, plan.head_dim, device=plan.device,
+                           softmax_scale=plan.softmax_scale, flags=plan.flags & ~FLAG_ZERO_PROMPT_GRAD, n_lanes=plan.n_lanes,
+                           kv_splits=plan.kv_splits)
+                if max(sub.ws_fwd_bytes, sub.ws_bwd_bytes) > self.out["ws"].numel():
+                    raise ValueError("workspace of the whole plan is smaller than a run's")
+                runs.append({"plan": sub, "r": (r0, acc), "p": (cu_p[g0], cu_p[g1 + 1]),
+                             "lse": torch.empty((plan.h_q, acc - r0), device=self.out["lse_r"].device, dtype=torch.float32),
+                             "ev_f_in": torch.cuda.Event(), "ev_b_in": torch.cuda.Event(),
+                             "ev_f_done": torch.cuda.Event(), "ev_b_done": torch.cuda.Event()})
+                b0, r0 = b + 1, acc
+        return runs
 
     def run(self, host_in, host_out):
+        if self.runs:
+            return self._run_chunked(host_in, host_out)
         plan, t, out = self.plan, self.t, self.out
         main = torch.cuda.current_stream()
         self.ev_start.record(main)                      # the device buffers are free once earlier work on `main` is done
@@ -328,6 +368,70 @@ class HostStep:
                 self.s_out.wait_event(ev)
                 for k in names:
                     host_out[k].copy_(out[k], non_blocking=True)
+            self.ev_out_end.record(self.s_out)
+        main.wait_event(self.ev_in_end)
+        main.wait_event(self.ev_out_end)
+
+    def _run_chunked(self, host_in, host_out):
+        plan, t, out, runs = self.plan, self.t, self.out, self.runs
+        main = torch.cuda.current_stream()
+        self.ev_start.record(main)
+        self.s_in.wait_event(self.ev_start)
+        self.s_out.wait_event(self.ev_start)
+        # ---- host -> device, in the order the calls can use them: the prompt's inputs and dO_P, then per run its q/k/v and dO
+        with torch.cuda.stream(self.s_in):
+            for k in ("q_p", "k_p", "v_p"):
+                t[k].copy_(host_in[k], non_blocking=True)
+            self.ev_in[0].record(self.s_in)
+            t["do_p"].copy_(host_in["do_p"], non_blocking=True)
+            self.ev_in[3].record(self.s_in)
+            for run in runs:
+                a, b = run["r"]
+                for k in ("q_r", "k_r", "v_r"):
+                    t[k][a:b].copy_(host_in[k][a:b], non_blocking=True)
+                run["ev_f_in"].record(self.s_in)
+                t["do_r"][a:b].copy_(host_in["do_r"][a:b], non_blocking=True)
+                run["ev_b_in"].record(self.s_in)
+            self.ev_in_end.record(self.s_in)
+        # ---- the calls.  The prompt-KV accumulators are sums (Eq. 2 plus the prefill's own part): with no bf16 copy of
+        # them asked for, the prefill backward may add its part first, so that dQ_P leaves while the replay runs compute.
+        if plan.flags & FLAG_ZERO_PROMPT_GRAD:      # the runs' plans do not clear: each ADDS its share of Eq. 2's sum
+            out["dk_p"].zero_()
+            out["dv_p"].zero_()
+        main.wait_event(self.ev_in[0])
+        plan.prefill_fwd(t["q_p"], t["k_p"], t["v_p"], out["o_p"], out["lse_p"], out["ws"])
+        self.ev_done[0].record(main)
+        main.wait_event(self.ev_in[3])
+        plan.prefill_bwd(t["q_p"], t["k_p"], t["v_p"], out["o_p"], out["lse_p"], t["do_p"], out["dk_p"], out["dv_p"], out["dq_p"],
+                         None, None, out["ws"])      # (adds its share; it never clears the accumulators)
+        self.ev_done[3].record(main)
+        for run in runs:
+            sub, (a, b), (pa, pb) = run["plan"], run["r"], run["p"]
+            kp, vp = t["k_p"][pa:pb], t["v_p"][pa:pb]
+            main.wait_event(run["ev_f_in"])
+            sub.replay_fwd(t["q_r"][a:b], t["k_r"][a:b], t["v_r"][a:b], kp, vp, out["o_r"][a:b], run["lse"], out["ws"])
+            out["lse_r"][:, a:b].copy_(run["lse"], non_blocking=True)     # LSE is head-major: a run's columns are strided
+            run["ev_f_done"].record(main)
+            main.wait_event(run["ev_b_in"])
+            sub.replay_bwd(t["q_r"][a:b], t["k_r"][a:b], t["v_r"][a:b], kp, vp, out["o_r"][a:b], run["lse"], t["do_r"][a:b],
+                           out["dq_r"][a:b], out["dk_r"][a:b], out["dv_r"][a:b], out["dk_p"][pa:pb], out["dv_p"][pa:pb], out["ws"])
+            run["ev_b_done"].record(main)
+        # ---- device -> host, each result as soon as its call is done
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.ev_done[0])
+            for k in ("o_p", "lse_p"):
+                host_out[k].copy_(out[k], non_blocking=True)
+            self.s_out.wait_event(self.ev_done[3])
+            host_out["dq_p"].copy_(out["dq_p"], non_blocking=True)
+            for run in runs:
+                a, b = run["r"]
+                self.s_out.wait_event(run["ev_f_done"])
+                host_out["o_r"][a:b].copy_(out["o_r"][a:b], non_blocking=True)
+                self.s_out.wait_event(run["ev_b_done"])
+                for k in ("dq_r", "dk_r", "dv_r"):
+                    host_out[k][a:b].copy_(out[k][a:b], non_blocking=True)
+            for k in ("lse_r", "dk_p", "dv_p"):
+                host_out[k].copy_(out[k], non_blocking=True)
             self.ev_out_end.record(self.s_out)
         main.wait_event(self.ev_in_end)
         main.wait_event(self.ev_out_end)

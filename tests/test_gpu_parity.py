@@ -195,6 +195,34 @@ def test_host_step_with_overlapped_copies_is_bitwise_the_plain_step(B):
         assert np.array_equal(v.float().numpy().astype(np.float64), plain[k]), k
 
 
+@pytest.mark.parametrize("chunks", [2, 3, 7])
+def test_host_step_in_runs_of_branches(B, chunks):
+    """HostStep with the response branches cut into runs (each with a plan of its own, forward and backward per run, the
+    copies of the next run under the kernels of this one): every result bit for bit the plain step's except the prompt-KV
+    accumulators, which take one addition per run instead of one per call (Eq. 2 associated differently): those against
+    the oracle, and against the plain step to fp32 rounding."""
+    w = _wl("hoststep-runs", [700, 130, 64], [[300, 150, 420], [257], [129, 65]], 8, 2, 96, 73)
+    t_cpu = wl.make_tensors(w)
+    plain, plan = pu.run_gpu(B, w, t_cpu, flags=B.FLAG_ZERO_PROMPT_GRAD)
+    dev_in = {k: torch.zeros_like(v, device="cuda") for k, v in t_cpu.items()}
+    out = B.alloc_outputs(plan)
+    host_in = {k: v.pin_memory() for k, v in t_cpu.items()}
+    host_out = {k: torch.full(v.shape, float("nan"), dtype=v.dtype).pin_memory() for k, v in out.items() if k != "ws"}
+    step = B.HostStep(plan, dev_in, out, chunks=chunks)
+    assert len(step.runs) == min(chunks, 6) and step.runs[0]["r"][0] == 0 and step.runs[-1]["r"][1] == plan.total_r
+    for _ in range(2):
+        step.run(host_in, host_out)
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0) and all(r["plan"].device_status() == (0, 0) for r in step.runs)
+    got = {k: v.float().numpy().astype(np.float64) for k, v in host_out.items()}
+    for k in got:
+        if k not in ("dk_p", "dv_p"):
+            assert np.array_equal(got[k], plain[k]), k
+    for k in ("dk_p", "dv_p"):
+        assert np.abs(got[k] - plain[k]).max() <= 1e-5 * max(1.0, np.abs(plain[k]).max()), k
+    pu.assert_parity(got, pu.run_oracle(w, t_cpu))
+
+
 def test_cuda_graph_replay_is_bitwise_the_eager_step(B):
     """The four entry points capture into a CUDA graph (no allocation or synchronisation in the launch path)."""
     w = _wl("graph", [256], [[128] * 4], 4, 4, 64, 61)
